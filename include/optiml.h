@@ -1,0 +1,145 @@
+/*
+ * optiml.h -- C ABI of the fused GEMM + bias + activation library for NVIDIA B200
+ * (sm_100a):
+ *
+ *     Y = act(A . B + bias)
+ *
+ * The contraction is the matrix product of the paper's Prompts appendix, task 2
+ * ("Matrix Multiplication": A is M x K, B is K x N, C = A x B is M x N), stored as
+ * in its matmul case study, "Common setup": every matrix dense and row-major,
+ * element (r, c) of an R x C matrix at index r*C + c, so A[m*K + k], B[k*N + n],
+ * Y[m*N + n].  act = ReLU is max(0, x) as in the Prompts appendix, task 10.  The
+ * length-N bias (added to every row) and the tanh form of GELU,
+ *     GELU(x) = 0.5 x (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3))),
+ * have no counterpart in the paper; they are this library's problem statement.
+ *
+ * Arithmetic.  OPTIML_F32: fp32 inputs, fp32 products and sums on the plain FMA
+ * pipes (no TF32, no split-precision tensor-core emulation), fp32 output.
+ * OPTIML_BF16: bf16 inputs, exact products, fp32 accumulation, bias widened to
+ * fp32, activation in fp32, one round-to-nearest-even to bf16 at the store.
+ * The summation order over k is unspecified but fixed for a given shape, device
+ * and variant: the same call gives the same bits every time.
+ *
+ * Threading / streams.  A handle is not thread-safe and serialises its own
+ * scratch memory in stream order: use one handle per stream.  Calls enqueue
+ * work on `stream` and return without synchronising unless stated otherwise.
+ *
+ * Errors are return codes; nothing aborts, traps or throws.
+ */
+#ifndef OPTIML_H_
+#define OPTIML_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct optiml_handle_s* optiml_handle_t;
+
+typedef enum {
+    OPTIML_OK = 0,
+    OPTIML_ERR_INVALID_ARG = 1, /* null pointer, non-positive dimension, bad enum         */
+    OPTIML_ERR_UNSUPPORTED = 2, /* forced variant cannot run this shape / dtype           */
+    OPTIML_ERR_ALIGNMENT = 3,   /* a device pointer is not aligned to its element size    */
+    OPTIML_ERR_ARCH = 4,        /* device is not compute capability 10.0                  */
+    OPTIML_ERR_ALLOC = 5,       /* device or host allocation failed                       */
+    OPTIML_ERR_CUDA = 6,        /* a CUDA runtime / driver call failed                    */
+    OPTIML_ERR_TIMEOUT = 7      /* a bounded on-device wait gave up (see get_last_status) */
+} optiml_status_t;
+
+typedef enum { OPTIML_F32 = 0, OPTIML_BF16 = 1 } optiml_dtype_t;
+
+typedef enum { OPTIML_ACT_NONE = 0, OPTIML_ACT_RELU = 1, OPTIML_ACT_GELU_TANH = 2 } optiml_act_t;
+
+/* Kernel variants the shape-based dispatcher chooses between. */
+typedef enum {
+    OPTIML_VARIANT_AUTO = -1,
+    OPTIML_VARIANT_GENERIC = 0,     /* predicated FMA tiles: any shape, any alignment, both dtypes      */
+    OPTIML_VARIANT_F32_TILED = 1,   /* fp32 FMA tiles, 128-bit loads: needs N % 4 == 0 and K % 4 == 0    */
+    OPTIML_VARIANT_GEMV_SPLITK = 2, /* bf16, M <= 4: split-K streaming with 128-bit loads, N % 8 == 0    */
+    OPTIML_VARIANT_SKINNY_UMMA = 3, /* bf16, M <= 128: stream-K over B with tcgen05 (N is the MMA M dim) */
+    OPTIML_VARIANT_UMMA = 4,        /* bf16: persistent TMA + tcgen05 + TMEM tiles, N % 8 == K % 8 == 0  */
+    OPTIML_VARIANT_COUNT = 5
+} optiml_variant_t;
+
+/*
+ * Create a handle on CUDA device `device` (host call).  Checks that the device is
+ * compute capability 10.0 (else OPTIML_ERR_ARCH), and allocates the handle's
+ * device scratch: split-K partial sums, arrival counters and a status word, about
+ * 40 MiB.  The calling thread's current device is left unchanged.
+ */
+optiml_status_t optiml_create(optiml_handle_t* out, int device);
+
+/* Free the handle and its scratch.  Synchronises the device first.  NULL is OK. */
+optiml_status_t optiml_destroy(optiml_handle_t h);
+
+/*
+ * Y = act(A . B + bias), enqueued on `stream` (a cudaStream_t; NULL = default
+ * stream).  Definition: header comment above (Prompts appendix task 2 and task 10;
+ * matmul case study, "Common setup").
+ *
+ *   A     device, M*K elements of dtype, row-major          read only
+ *   B     device, K*N elements of dtype, row-major          read only
+ *   bias  device, N elements of dtype, or NULL for zeros    read only
+ *   Y     device, M*N elements of dtype, row-major          written once; must not
+ *         overlap A, B or bias
+ *   M, N, K  >= 1, each <= 2^31 - 1
+ *
+ * All four buffers stay owned by the caller and must stay valid until the work
+ * has run; the library keeps no reference after that.  Pointers must be aligned
+ * to the element size; the fast variants also need 16-byte aligned pointers and
+ * N, K multiples of 8 (bf16) or 4 (fp32) -- other shapes run on the generic
+ * variant, never on the CPU.  Inputs must be finite.  Scratch use is serialised
+ * on `stream`; do not use one handle on two streams at once.
+ *
+ * Returns OPTIML_OK once the work is enqueued; INVALID_ARG / ALIGNMENT before
+ * anything is launched; CUDA if a launch failed.  A bounded on-device wait that
+ * gave up is reported by optiml_get_last_status after synchronisation.
+ */
+optiml_status_t optiml_gemm_epilogue(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y,
+                                     int64_t M, int64_t N, int64_t K, optiml_dtype_t dtype, optiml_act_t act,
+                                     void* stream);
+
+/*
+ * Same operation with HOST buffers (same shapes and dtype as above): copies A, B
+ * and bias to device staging memory owned by the handle (grown on demand, which
+ * allocates), runs optiml_gemm_epilogue on `stream`, copies Y back and
+ * synchronises `stream` before returning.  Pinned host memory makes the copies
+ * asynchronous with respect to the host until that final synchronisation.
+ */
+optiml_status_t optiml_gemm_epilogue_host(optiml_handle_t h, const void* A_host, const void* B_host,
+                                          const void* bias_host, void* Y_host, int64_t M, int64_t N, int64_t K,
+                                          optiml_dtype_t dtype, optiml_act_t act, void* stream);
+
+/*
+ * Read the device-written status word (synchronises the device): OPTIML_OK, or
+ * OPTIML_ERR_TIMEOUT if any kernel of this handle gave up a bounded wait since the
+ * last call of this function; the word is cleared.  A call that reported a
+ * time-out has left Y undefined.
+ */
+optiml_status_t optiml_get_last_status(optiml_handle_t h);
+
+/* Force one variant for later calls (tests, profiling), or OPTIML_VARIANT_AUTO to
+ * give the choice back to the dispatcher.  A forced variant that cannot run a
+ * shape makes optiml_gemm_epilogue return OPTIML_ERR_UNSUPPORTED. */
+optiml_status_t optiml_force_variant(optiml_handle_t h, optiml_variant_t v);
+
+/* Variant the dispatcher would run for this problem (honours a forced variant;
+ * pointers are assumed 16-byte aligned), or -1 on bad arguments. */
+int optiml_select_variant(optiml_handle_t h, int64_t M, int64_t N, int64_t K, optiml_dtype_t dtype);
+
+/* Number of kernels launched by this handle since it was created. */
+int64_t optiml_launch_count(optiml_handle_t h);
+
+/* Static strings; never NULL. */
+const char* optiml_status_string(optiml_status_t s);
+const char* optiml_variant_name(int variant);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int optiml_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OPTIML_H_ */

@@ -1,0 +1,488 @@
+// C ABI of the library (include/optiml.h): handle, argument checks, the shape-based
+// dispatcher and the kernel launches.  Host code only touches scalars and pointers;
+// every arithmetic step of Y = act(A.B + bias) runs in the kernels included below.
+#include "../../include/optiml.h"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "kernel_f32.cuh"
+#include "kernel_gemv.cuh"
+#include "kernel_generic.cuh"
+#include "kernel_skinny.cuh"
+#include "kernel_umma.cuh"
+
+using namespace optiml;
+
+namespace {
+
+constexpr int kVersion = 10000 * 0 + 100 * 1 + 0;
+constexpr size_t kPartialBytes = (size_t)32 << 20;   // split-K / stream-K partial sums
+constexpr int kNumCounters = 1 << 16;                 // one arrival counter per column block / tile
+constexpr int kMapCache = 16;
+
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct MapEntry {
+    const void* ptr = nullptr;
+    uint64_t rows = 0, cols = 0;
+    uint32_t box_rows = 0, box_cols = 0;
+    CUtensorMap map;
+    bool valid = false;
+};
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+struct optiml_handle_s {
+    int device = 0;
+    int num_sms = 0;
+    float* partials = nullptr;
+    unsigned int* counters = nullptr;
+    int* status = nullptr;
+    int forced = OPTIML_VARIANT_AUTO;
+    int64_t launches = 0;
+    bool log = false;
+    encode_tiled_fn encode = nullptr;
+    MapEntry maps[kMapCache];
+    int next_map = 0;
+    void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
+    size_t stage_bytes[4] = {0, 0, 0, 0};
+};
+
+namespace {
+
+// ---------------------------------------------------------------- tensor maps
+
+// Row-major bf16 matrix [rows][cols] -> 2-D tiled map with a {box_cols, box_rows} box and
+// 128-byte swizzle (box_cols * 2 bytes == 128).  Cached by (pointer, shape, box).
+const CUtensorMap* get_map(optiml_handle_t h, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                           uint32_t box_cols) {
+    for (int i = 0; i < kMapCache; ++i) {
+        MapEntry& e = h->maps[i];
+        if (e.valid && e.ptr == ptr && e.rows == rows && e.cols == cols && e.box_rows == box_rows &&
+            e.box_cols == box_cols)
+            return &e.map;
+    }
+    MapEntry& e = h->maps[h->next_map];
+    h->next_map = (h->next_map + 1) % kMapCache;
+    e.valid = false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = h->encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box,
+                           estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return nullptr;
+    e.ptr = ptr;
+    e.rows = rows;
+    e.cols = cols;
+    e.box_rows = box_rows;
+    e.box_cols = box_cols;
+    e.valid = true;
+    return &e.map;
+}
+
+// ---------------------------------------------------------------- dispatcher
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+bool variant_supports(int v, int64_t M, int64_t N, int64_t K, int dtype, bool al16) {
+    switch (v) {
+    case OPTIML_VARIANT_GENERIC:
+        return true;
+    case OPTIML_VARIANT_F32_TILED:
+        return dtype == OPTIML_F32 && N % 4 == 0 && K % 4 == 0 && al16;
+    case OPTIML_VARIANT_GEMV_SPLITK:
+        return dtype == OPTIML_BF16 && M <= 4 && N % 8 == 0 && al16 && ceil_div64(N, kGemvCols) <= kNumCounters;
+    case OPTIML_VARIANT_SKINNY_UMMA:
+        return dtype == OPTIML_BF16 && M <= 128 && N % 8 == 0 && K % 8 == 0 && al16 &&
+               ceil_div64(N, 128) <= kNumCounters;
+    case OPTIML_VARIANT_UMMA:
+        return dtype == OPTIML_BF16 && N % 8 == 0 && K % 8 == 0 && al16 &&
+               ceil_div64(M, UmmaCfg::BM) * ceil_div64(N, UmmaCfg::BN) < (int64_t)1 << 31;
+    default:
+        return false;
+    }
+}
+
+// Shape-based choice.  fp32 goes to the FMA tiles.  bf16: M <= 4 is a pure stream over B
+// (CUDA-core split-K), M <= 64 is still bandwidth-bound but needs tensor-core MACs
+// (stream-K tcgen05 with N as the MMA M dimension), larger M is compute-bound.
+int choose_variant(optiml_handle_t h, int64_t M, int64_t N, int64_t K, int dtype, bool al16) {
+    if (h->forced != OPTIML_VARIANT_AUTO) return h->forced;
+    if (dtype == OPTIML_F32)
+        return variant_supports(OPTIML_VARIANT_F32_TILED, M, N, K, dtype, al16) ? OPTIML_VARIANT_F32_TILED
+                                                                                 : OPTIML_VARIANT_GENERIC;
+    if (M <= 4 && variant_supports(OPTIML_VARIANT_GEMV_SPLITK, M, N, K, dtype, al16)) return OPTIML_VARIANT_GEMV_SPLITK;
+    if (M <= 64 && variant_supports(OPTIML_VARIANT_SKINNY_UMMA, M, N, K, dtype, al16)) return OPTIML_VARIANT_SKINNY_UMMA;
+    if (variant_supports(OPTIML_VARIANT_UMMA, M, N, K, dtype, al16)) return OPTIML_VARIANT_UMMA;
+    return OPTIML_VARIANT_GENERIC;
+}
+
+// ---------------------------------------------------------------- launches
+
+template <typename T>
+optiml_status_t launch_generic(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M,
+                               int N, int K, int act, cudaStream_t st) {
+    const int64_t tiles = ceil_div64(M, kGenBM) * ceil_div64(N, kGenBN);
+    if (tiles >= (int64_t)1 << 31) return OPTIML_ERR_UNSUPPORTED;
+    gemm_generic_kernel<T><<<(unsigned)tiles, kGenThreads, 0, st>>>((const T*)A, (const T*)B, (const T*)bias, (T*)Y, M,
+                                                                     N, K, act);
+    h->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+template <int BM, int BN, int TM, int TN, int KS>
+optiml_status_t launch_f32_cfg(optiml_handle_t h, const float* A, const float* B, const float* bias, float* Y, int M,
+                               int N, int K, int act, cudaStream_t st) {
+    using C = F32Cfg<BM, BN, TM, TN, KS>;
+    const int64_t tiles = ceil_div64(M, BM) * ceil_div64(N, BN);
+    if (tiles >= (int64_t)1 << 31) return OPTIML_ERR_UNSUPPORTED;
+    const size_t smem = C::kSmemFloats * sizeof(float);
+    switch (act) {
+    case OPTIML_ACT_RELU:
+        gemm_f32_tiled_kernel<BM, BN, TM, TN, KS, kActRelu><<<(unsigned)tiles, C::kThreads, smem, st>>>(A, B, bias, Y, M, N, K);
+        break;
+    case OPTIML_ACT_GELU_TANH:
+        gemm_f32_tiled_kernel<BM, BN, TM, TN, KS, kActGeluTanh><<<(unsigned)tiles, C::kThreads, smem, st>>>(A, B, bias, Y, M, N, K);
+        break;
+    default:
+        gemm_f32_tiled_kernel<BM, BN, TM, TN, KS, kActNone><<<(unsigned)tiles, C::kThreads, smem, st>>>(A, B, bias, Y, M, N, K);
+        break;
+    }
+    h->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+// Largest tile that still gives every SM a CTA; small problems take 32x32 tiles with the
+// K loop split four ways inside the CTA.
+optiml_status_t launch_f32(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
+                           int K, int act, cudaStream_t st) {
+    const float *a = (const float*)A, *b = (const float*)B, *bi = (const float*)bias;
+    float* y = (float*)Y;
+    if (ceil_div64(M, 128) * ceil_div64(N, 128) >= h->num_sms)
+        return launch_f32_cfg<128, 128, 8, 8, 1>(h, a, b, bi, y, M, N, K, act, st);
+    if (ceil_div64(M, 64) * ceil_div64(N, 64) >= h->num_sms)
+        return launch_f32_cfg<64, 64, 4, 4, 1>(h, a, b, bi, y, M, N, K, act, st);
+    return launch_f32_cfg<32, 32, 4, 4, 4>(h, a, b, bi, y, M, N, K, act, st);
+}
+
+template <int MR>
+void launch_gemv_mr(const void* A, const void* B, const void* bias, void* Y, int M, int N, int K, int act, dim3 grid,
+                    float* partials, unsigned int* counters, cudaStream_t st) {
+    gemv_splitk_kernel<MR><<<grid, kGemvThreads, 0, st>>>((const __nv_bfloat16*)A, (const __nv_bfloat16*)B,
+                                                          (const __nv_bfloat16*)bias, (__nv_bfloat16*)Y, M, N, K, act,
+                                                          partials, counters);
+}
+
+optiml_status_t launch_gemv(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
+                            int K, int act, cudaStream_t st) {
+    const int MR = M == 1 ? 1 : (M == 2 ? 2 : 4);
+    const int64_t col_blocks = ceil_div64(N, kGemvCols);
+    // K slices: fill every SM with two CTAs in one wave, keep at least 64 rows per slice,
+    // stay inside the scratch and the 65535 limit of gridDim.y.
+    int64_t S = (2 * (int64_t)h->num_sms) / col_blocks;
+    if (S > K / 64) S = K / 64;
+    const int64_t per_slice = (int64_t)MR * kGemvCols * sizeof(float);
+    if (S * col_blocks * per_slice > (int64_t)kPartialBytes) S = kPartialBytes / (col_blocks * per_slice);
+    if (S > 65535) S = 65535;
+    if (S < 1) S = 1;
+    dim3 grid((unsigned)col_blocks, (unsigned)S);
+    if (MR == 1) launch_gemv_mr<1>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
+    else if (MR == 2) launch_gemv_mr<2>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
+    else launch_gemv_mr<4>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
+    h->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+template <int MP>
+optiml_status_t launch_skinny_mp(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M,
+                                 int N, int K, int act, cudaStream_t st) {
+    using C = SkinnyCfg<MP>;
+    const CUtensorMap* ma = get_map(h, A, (uint64_t)M, (uint64_t)K, MP, 64);
+    const CUtensorMap* mb = get_map(h, B, (uint64_t)K, (uint64_t)N, 64, 64);
+    if (!ma || !mb) return OPTIML_ERR_CUDA;
+    const int64_t units = ceil_div64(N, C::BN) * ceil_div64(K, C::BK);
+    int G = h->num_sms;
+    if (units < G) G = (int)units;
+    // two scratch slots per CTA
+    if ((size_t)2 * G * C::kSlotFloats * sizeof(float) > kPartialBytes) return OPTIML_ERR_UNSUPPORTED;
+    gemm_skinny_umma_kernel<MP><<<G, C::kThreads, C::kSmemBytes, st>>>(*ma, *mb, (const __nv_bfloat16*)bias,
+                                                                       (__nv_bfloat16*)Y, M, N, K, act, h->partials,
+                                                                       h->counters, h->status);
+    h->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+optiml_status_t launch_skinny(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
+                              int K, int act, cudaStream_t st) {
+    if (M <= 16) return launch_skinny_mp<16>(h, A, B, bias, Y, M, N, K, act, st);
+    if (M <= 32) return launch_skinny_mp<32>(h, A, B, bias, Y, M, N, K, act, st);
+    if (M <= 64) return launch_skinny_mp<64>(h, A, B, bias, Y, M, N, K, act, st);
+    return launch_skinny_mp<128>(h, A, B, bias, Y, M, N, K, act, st);
+}
+
+optiml_status_t launch_umma(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
+                            int K, int act, cudaStream_t st) {
+    using C = UmmaCfg;
+    const CUtensorMap* ma = get_map(h, A, (uint64_t)M, (uint64_t)K, C::BM, 64);
+    const CUtensorMap* mb = get_map(h, B, (uint64_t)K, (uint64_t)N, 64, 64);
+    if (!ma || !mb) return OPTIML_ERR_CUDA;
+    const int64_t tiles = ceil_div64(M, C::BM) * ceil_div64(N, C::BN);
+    const int grid = (int)(tiles < h->num_sms ? tiles : h->num_sms);
+    const __nv_bfloat16* bi = (const __nv_bfloat16*)bias;
+    __nv_bfloat16* y = (__nv_bfloat16*)Y;
+    switch (act) {
+    case OPTIML_ACT_RELU:
+        gemm_umma_kernel<kActRelu><<<grid, C::kThreads, C::kSmemBytes, st>>>(*ma, *mb, bi, y, M, N, K, h->status);
+        break;
+    case OPTIML_ACT_GELU_TANH:
+        gemm_umma_kernel<kActGeluTanh><<<grid, C::kThreads, C::kSmemBytes, st>>>(*ma, *mb, bi, y, M, N, K, h->status);
+        break;
+    default:
+        gemm_umma_kernel<kActNone><<<grid, C::kThreads, C::kSmemBytes, st>>>(*ma, *mb, bi, y, M, N, K, h->status);
+        break;
+    }
+    h->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+template <typename F>
+bool set_smem(F* fn, int bytes) {
+    return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+
+bool configure_kernels() {
+    bool ok = true;
+    ok &= set_smem(gemm_umma_kernel<kActNone>, UmmaCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma_kernel<kActRelu>, UmmaCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma_kernel<kActGeluTanh>, UmmaCfg::kSmemBytes);
+    ok &= set_smem(gemm_skinny_umma_kernel<16>, SkinnyCfg<16>::kSmemBytes);
+    ok &= set_smem(gemm_skinny_umma_kernel<32>, SkinnyCfg<32>::kSmemBytes);
+    ok &= set_smem(gemm_skinny_umma_kernel<64>, SkinnyCfg<64>::kSmemBytes);
+    ok &= set_smem(gemm_skinny_umma_kernel<128>, SkinnyCfg<128>::kSmemBytes);
+    return ok;
+}
+
+optiml_status_t check_args(optiml_handle_t h, const void* A, const void* B, const void* Y, int64_t M, int64_t N,
+                           int64_t K, int dtype, int act) {
+    if (!h || !A || !B || !Y) return OPTIML_ERR_INVALID_ARG;
+    if (M < 1 || N < 1 || K < 1 || M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return OPTIML_ERR_INVALID_ARG;
+    if (dtype != OPTIML_F32 && dtype != OPTIML_BF16) return OPTIML_ERR_INVALID_ARG;
+    if (act != OPTIML_ACT_NONE && act != OPTIML_ACT_RELU && act != OPTIML_ACT_GELU_TANH) return OPTIML_ERR_INVALID_ARG;
+    return OPTIML_OK;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------- exported entry points
+
+extern "C" {
+
+optiml_status_t optiml_create(optiml_handle_t* out, int device) {
+    if (!out) return OPTIML_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess) return OPTIML_ERR_CUDA;
+    if (device < 0 || device >= count) return OPTIML_ERR_INVALID_ARG;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return OPTIML_ERR_CUDA;
+    if (prop.major != 10 || prop.minor != 0) return OPTIML_ERR_ARCH;
+
+    optiml_handle_t h = new (std::nothrow) optiml_handle_s();
+    if (!h) return OPTIML_ERR_ALLOC;
+    h->device = device;
+    h->num_sms = prop.multiProcessorCount;
+    const char* lg = getenv("OPTIML_LOG");
+    h->log = lg && lg[0] == '1';
+
+    DeviceGuard guard(device);
+    cudaDriverEntryPointQueryResult qres;
+    void* fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess) {
+        delete h;
+        return OPTIML_ERR_CUDA;
+    }
+    h->encode = reinterpret_cast<encode_tiled_fn>(fn);
+
+    bool ok = cudaMalloc(&h->partials, kPartialBytes) == cudaSuccess;
+    ok = ok && cudaMalloc(&h->counters, kNumCounters * sizeof(unsigned int)) == cudaSuccess;
+    ok = ok && cudaMalloc(&h->status, sizeof(int)) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        optiml_destroy(h);
+        return OPTIML_ERR_ALLOC;
+    }
+    ok = cudaMemset(h->counters, 0, kNumCounters * sizeof(unsigned int)) == cudaSuccess;
+    ok = ok && cudaMemset(h->status, 0, sizeof(int)) == cudaSuccess;
+    ok = ok && configure_kernels();
+    ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        optiml_destroy(h);
+        return OPTIML_ERR_CUDA;
+    }
+    *out = h;
+    return OPTIML_OK;
+}
+
+optiml_status_t optiml_destroy(optiml_handle_t h) {
+    if (!h) return OPTIML_OK;
+    DeviceGuard guard(h->device);
+    cudaDeviceSynchronize();
+    cudaFree(h->partials);
+    cudaFree(h->counters);
+    cudaFree(h->status);
+    for (int i = 0; i < 4; ++i) cudaFree(h->stage[i]);
+    cudaGetLastError();
+    delete h;
+    return OPTIML_OK;
+}
+
+optiml_status_t optiml_gemm_epilogue(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y,
+                                     int64_t M, int64_t N, int64_t K, optiml_dtype_t dtype, optiml_act_t act,
+                                     void* stream) {
+    optiml_status_t s = check_args(h, A, B, Y, M, N, K, (int)dtype, (int)act);
+    if (s != OPTIML_OK) return s;
+    const uintptr_t es = dtype == OPTIML_F32 ? 4 : 2;
+    const uintptr_t all = reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B) |
+                          reinterpret_cast<uintptr_t>(bias) | reinterpret_cast<uintptr_t>(Y);
+    if (all & (es - 1)) return OPTIML_ERR_ALIGNMENT;
+    const bool al16 = aligned16(A) && aligned16(B) && aligned16(bias) && aligned16(Y);
+    const int v = choose_variant(h, M, N, K, (int)dtype, al16);
+    if (!variant_supports(v, M, N, K, (int)dtype, al16)) return OPTIML_ERR_UNSUPPORTED;
+    if (h->log)
+        fprintf(stderr, "[optiml] M=%lld N=%lld K=%lld dtype=%d act=%d -> %s\n", (long long)M, (long long)N,
+                (long long)K, (int)dtype, (int)act, optiml_variant_name(v));
+
+    DeviceGuard guard(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int m = (int)M, n = (int)N, k = (int)K;
+    switch (v) {
+    case OPTIML_VARIANT_F32_TILED:
+        return launch_f32(h, A, B, bias, Y, m, n, k, (int)act, st);
+    case OPTIML_VARIANT_GEMV_SPLITK:
+        return launch_gemv(h, A, B, bias, Y, m, n, k, (int)act, st);
+    case OPTIML_VARIANT_SKINNY_UMMA:
+        return launch_skinny(h, A, B, bias, Y, m, n, k, (int)act, st);
+    case OPTIML_VARIANT_UMMA:
+        return launch_umma(h, A, B, bias, Y, m, n, k, (int)act, st);
+    default:
+        return dtype == OPTIML_F32 ? launch_generic<float>(h, A, B, bias, Y, m, n, k, (int)act, st)
+                                   : launch_generic<__nv_bfloat16>(h, A, B, bias, Y, m, n, k, (int)act, st);
+    }
+}
+
+optiml_status_t optiml_gemm_epilogue_host(optiml_handle_t h, const void* A_host, const void* B_host,
+                                          const void* bias_host, void* Y_host, int64_t M, int64_t N, int64_t K,
+                                          optiml_dtype_t dtype, optiml_act_t act, void* stream) {
+    optiml_status_t s = check_args(h, A_host, B_host, Y_host, M, N, K, (int)dtype, (int)act);
+    if (s != OPTIML_OK) return s;
+    DeviceGuard guard(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t es = dtype == OPTIML_F32 ? 4 : 2;
+    const size_t need[4] = {(size_t)M * K * es, (size_t)K * N * es, (size_t)N * es, (size_t)M * N * es};
+    for (int i = 0; i < 4; ++i) {
+        if (h->stage_bytes[i] >= need[i]) continue;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return OPTIML_ERR_CUDA;   // earlier work may still use it
+        cudaFree(h->stage[i]);
+        h->stage[i] = nullptr;
+        h->stage_bytes[i] = 0;
+        if (cudaMalloc(&h->stage[i], need[i]) != cudaSuccess) {
+            cudaGetLastError();
+            return OPTIML_ERR_ALLOC;
+        }
+        h->stage_bytes[i] = need[i];
+    }
+    bool ok = cudaMemcpyAsync(h->stage[0], A_host, need[0], cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(h->stage[1], B_host, need[1], cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (bias_host) ok = ok && cudaMemcpyAsync(h->stage[2], bias_host, need[2], cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (!ok) return OPTIML_ERR_CUDA;
+    s = optiml_gemm_epilogue(h, h->stage[0], h->stage[1], bias_host ? h->stage[2] : nullptr, h->stage[3], M, N, K, dtype,
+                             act, stream);
+    if (s != OPTIML_OK) return s;
+    ok = cudaMemcpyAsync(Y_host, h->stage[3], need[3], cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+    return ok ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+optiml_status_t optiml_get_last_status(optiml_handle_t h) {
+    if (!h) return OPTIML_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    int word = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return OPTIML_ERR_CUDA;
+    if (cudaMemcpy(&word, h->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return OPTIML_ERR_CUDA;
+    if (word != kDevOk) {
+        // a kernel that gave up may have left arrival counters half way: re-arm everything
+        cudaMemset(h->status, 0, sizeof(int));
+        cudaMemset(h->counters, 0, kNumCounters * sizeof(unsigned int));
+        cudaDeviceSynchronize();
+        return OPTIML_ERR_TIMEOUT;
+    }
+    return OPTIML_OK;
+}
+
+optiml_status_t optiml_force_variant(optiml_handle_t h, optiml_variant_t v) {
+    if (!h || (int)v < OPTIML_VARIANT_AUTO || (int)v >= OPTIML_VARIANT_COUNT) return OPTIML_ERR_INVALID_ARG;
+    h->forced = (int)v;
+    return OPTIML_OK;
+}
+
+int optiml_select_variant(optiml_handle_t h, int64_t M, int64_t N, int64_t K, optiml_dtype_t dtype) {
+    if (!h || M < 1 || N < 1 || K < 1 || (dtype != OPTIML_F32 && dtype != OPTIML_BF16)) return -1;
+    return choose_variant(h, M, N, K, (int)dtype, true);
+}
+
+int64_t optiml_launch_count(optiml_handle_t h) { return h ? h->launches : -1; }
+
+const char* optiml_status_string(optiml_status_t s) {
+    switch (s) {
+    case OPTIML_OK: return "ok";
+    case OPTIML_ERR_INVALID_ARG: return "invalid argument";
+    case OPTIML_ERR_UNSUPPORTED: return "shape or dtype not supported by the forced variant";
+    case OPTIML_ERR_ALIGNMENT: return "pointer not aligned to its element size";
+    case OPTIML_ERR_ARCH: return "device is not compute capability 10.0 (B200)";
+    case OPTIML_ERR_ALLOC: return "allocation failed";
+    case OPTIML_ERR_CUDA: return "CUDA call failed";
+    case OPTIML_ERR_TIMEOUT: return "a bounded on-device wait gave up";
+    default: return "unknown status";
+    }
+}
+
+const char* optiml_variant_name(int variant) {
+    switch (variant) {
+    case OPTIML_VARIANT_AUTO: return "auto";
+    case OPTIML_VARIANT_GENERIC: return "generic_fma";
+    case OPTIML_VARIANT_F32_TILED: return "f32_tiled_fma";
+    case OPTIML_VARIANT_GEMV_SPLITK: return "gemv_splitk_stream";
+    case OPTIML_VARIANT_SKINNY_UMMA: return "skinny_streamk_tcgen05";
+    case OPTIML_VARIANT_UMMA: return "persistent_tcgen05";
+    default: return "unknown";
+    }
+}
+
+int optiml_version(void) { return kVersion; }
+
+}  // extern "C"

@@ -1,0 +1,287 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the
+same seeded inputs -- element by element at sizes the oracle finishes in seconds (several
+tiles plus ragged tails, every variant forced in turn), bit-exact on integer-valued
+inputs, and on sampled outputs at the five full-size workloads."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle
+from paper_2602_12305_b200 import binding, synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+F32, BF16 = synth.F32, synth.BF16
+NONE, RELU, GELU = synth.ACT_NONE, synth.ACT_RELU, synth.ACT_GELU_TANH
+V = binding
+
+
+@pytest.fixture(scope="module")
+def handle():
+    h = binding.Handle(0)
+    yield h
+    h.destroy()
+
+
+@pytest.fixture(autouse=True)
+def _auto_variant(handle):
+    handle.force_variant(V.VARIANT_AUTO)
+    yield
+    handle.force_variant(V.VARIANT_AUTO)
+
+
+def parity(handle, case, variant=None, what=""):
+    if variant is not None:
+        handle.force_variant(variant)
+    bits, y = H.run_case(handle, case)
+    H.check_tolerance(y, H.oracle_full(case), case.dtype, what or f"{case.name} {case.M}x{case.N}x{case.K}")
+    return bits
+
+
+# ---------------------------------------------------------------- every variant, small and ragged shapes
+
+@pytest.mark.parametrize("name,M,N,K", [("c1", 1, 1, 1), ("c1", 3, 5, 7), ("c1", 65, 130, 33), ("c1", 200, 300, 150),
+                                         ("c4", 1, 1, 1), ("c4", 3, 5, 7), ("c4", 65, 130, 33), ("c2", 1, 257, 1000)])
+@pytest.mark.parametrize("act", [NONE, RELU, GELU])
+def test_generic_variant(handle, name, M, N, K, act):
+    parity(handle, synth.make_case(name, M=M, N=N, K=K, act=act), V.VARIANT_GENERIC)
+
+
+@pytest.mark.parametrize("M,N,K", [(256, 256, 256), (8, 12, 20), (260, 132, 516), (37, 64, 4), (130, 260, 1028),
+                                   (1000, 1280, 96),      # >= 148 tiles of 64x64
+                                   (1664, 1536, 72)])     # >= 148 tiles of 128x128
+@pytest.mark.parametrize("act", [RELU, GELU])
+def test_f32_tiled_variant(handle, M, N, K, act):
+    parity(handle, synth.make_case("c1", M=M, N=N, K=K, act=act), V.VARIANT_F32_TILED)
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 512, 1024), (1, 264, 100), (2, 1032, 333), (3, 520, 777), (4, 8192, 300),
+                                   (1, 8, 1), (4, 40000, 64)])
+@pytest.mark.parametrize("act", [NONE, GELU])
+def test_gemv_variant(handle, M, N, K, act):
+    parity(handle, synth.make_case("c2", M=M, N=N, K=K, act=act), V.VARIANT_GEMV_SPLITK)
+
+
+@pytest.mark.parametrize("M,N,K", [(16, 1160, 1096),     # 180 units over 148 CTAs: tiles split mid-K
+                                   (16, 20480, 64),      # one K block per tile: every segment whole
+                                   (1, 1024, 2048), (5, 136, 8), (17, 392, 520), (33, 1288, 264), (64, 2056, 712),
+                                   (100, 520, 1096), (128, 1160, 328)])
+@pytest.mark.parametrize("act", [RELU, GELU])
+def test_skinny_variant(handle, M, N, K, act):
+    parity(handle, synth.make_case("c3", M=M, N=N, K=K, act=act), V.VARIANT_SKINNY_UMMA)
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (128, 256, 512), (300, 520, 200), (130, 264, 72), (1, 8, 8),
+                                   (1024, 1024, 512),
+                                   (2048, 4096, 128)])   # 256 tiles: more than one tile per CTA
+@pytest.mark.parametrize("act", [RELU, GELU])
+def test_umma_variant(handle, M, N, K, act):
+    parity(handle, synth.make_case("c4", M=M, N=N, K=K, act=act), V.VARIANT_UMMA)
+
+
+def test_null_bias_and_act_none(handle):
+    for variant, name, shape in ((V.VARIANT_F32_TILED, "c1", (64, 64, 64)), (V.VARIANT_GEMV_SPLITK, "c2", (1, 512, 512)),
+                                 (V.VARIANT_SKINNY_UMMA, "c3", (16, 512, 512)), (V.VARIANT_UMMA, "c4", (256, 512, 256)),
+                                 (V.VARIANT_GENERIC, "c4", (50, 60, 70))):
+        c = synth.make_case(name, M=shape[0], N=shape[1], K=shape[2], act=NONE)
+        c.bias = None
+        parity(handle, c, variant)
+
+
+# ---------------------------------------------------------------- integer-valued inputs: bit-exact
+
+@pytest.mark.parametrize("variant,dtype,M,N,K", [
+    (V.VARIANT_GENERIC, F32, 70, 90, 300), (V.VARIANT_GENERIC, BF16, 70, 90, 300),
+    (V.VARIANT_F32_TILED, F32, 96, 160, 512), (V.VARIANT_GEMV_SPLITK, BF16, 1, 1024, 4096),
+    (V.VARIANT_GEMV_SPLITK, BF16, 4, 520, 1000), (V.VARIANT_SKINNY_UMMA, BF16, 16, 1160, 1096),
+    (V.VARIANT_SKINNY_UMMA, BF16, 48, 648, 2048), (V.VARIANT_UMMA, BF16, 384, 776, 1024)])
+@pytest.mark.parametrize("act", [NONE, RELU])
+def test_integer_inputs_are_bit_exact(handle, variant, dtype, M, N, K, act):
+    c = synth.integer_case(M, N, K, dtype, act, seed=11)
+    handle.force_variant(variant)
+    bits, _ = H.run_case(handle, c)
+    H.check_bit_exact(bits, H.oracle_full(c), dtype, f"{binding.variant_name(variant)} {M}x{N}x{K}")
+
+
+def test_permutation_B_on_the_tensor_core_path(handle):
+    # B = permutation matrix: Y's columns are A's columns permuted, exactly (catches a
+    # transposed or mis-swizzled operand on the MMA paths).
+    M, K = 256, 512
+    c = synth.integer_case(M, K, K, BF16, NONE, seed=2)
+    perm = np.random.default_rng(0).permutation(K)
+    Bm = np.zeros((K, K))
+    Bm[perm, np.arange(K)] = 1.0
+    c.B = synth.round_to_bf16_bits(Bm).reshape(-1)
+    c.bias = None
+    for variant in (V.VARIANT_UMMA, V.VARIANT_SKINNY_UMMA, V.VARIANT_GENERIC):
+        if variant == V.VARIANT_SKINNY_UMMA:
+            c2 = synth.Case("perm", 64, K, K, BF16, NONE, c.A[:64 * K], c.B, None)
+        else:
+            c2 = c
+        handle.force_variant(variant)
+        _, y = H.run_case(handle, c2)
+        A = oracle.widen(c2.A, BF16).reshape(c2.M, K)
+        assert np.array_equal(y, A[:, perm])
+
+
+# ---------------------------------------------------------------- the five full-size workloads
+
+def sample_indices(n, tile, count, seed):
+    """Indices covering every residue modulo `tile`, the first and last tile, plus random ones."""
+    rng = np.random.default_rng(seed)
+    base = (np.arange(tile) + tile * rng.integers(0, max(1, n // tile), tile)) % n
+    extra = rng.integers(0, n, max(0, count - tile))
+    edge = np.array([0, 1, n - 2, n - 1, min(n - 1, tile - 1), min(n - 1, tile)])
+    return np.unique(np.concatenate([base, extra, edge]))
+
+
+def test_c1_full(handle):
+    c = synth.make_case("c1")
+    assert handle.select_variant(c.M, c.N, c.K, c.dtype) == V.VARIANT_F32_TILED
+    parity(handle, c)
+
+
+@pytest.mark.parametrize("sigma", [None, 8192 ** -0.5])
+def test_c2_full(handle, sigma):
+    c = synth.make_case("c2", sigma=sigma)
+    assert handle.select_variant(c.M, c.N, c.K, c.dtype) in (V.VARIANT_GEMV_SPLITK, V.VARIANT_SKINNY_UMMA)
+    parity(handle, c)
+    parity(handle, c, V.VARIANT_GEMV_SPLITK)
+    parity(handle, c, V.VARIANT_SKINNY_UMMA)
+
+
+def test_c3_full(handle):
+    c = synth.make_case("c3")
+    assert handle.select_variant(c.M, c.N, c.K, c.dtype) == V.VARIANT_SKINNY_UMMA
+    bits = parity(handle, c)
+    bits2, _ = H.run_case(handle, c)
+    assert np.array_equal(bits, bits2), "stream-K reduction is not reproducible"
+
+
+@pytest.mark.parametrize("name", ["c4", "c5"])
+def test_c4_c5_sampled(handle, name):
+    c = synth.make_case(name)
+    assert handle.select_variant(c.M, c.N, c.K, c.dtype) == V.VARIANT_UMMA
+    bits, y = H.run_case(handle, c)
+    rows = sample_indices(c.M, 128, 160, 1)
+    cols = sample_indices(c.N, 256, 288, 2)
+    ref = oracle.gemm_epilogue_sampled(c.A, c.B, c.bias, c.M, c.N, c.K, c.dtype, c.act, rows, cols)
+    H.check_tolerance(y[np.ix_(rows, cols)], ref, c.dtype, f"{name} sampled {len(rows)}x{len(cols)}")
+    # a few complete rows and columns as well
+    frows = np.array([0, c.M // 2 + 3, c.M - 1])
+    ref_r = oracle.gemm_epilogue_sampled(c.A, c.B, c.bias, c.M, c.N, c.K, c.dtype, c.act, frows, np.arange(c.N))
+    H.check_tolerance(y[frows], ref_r, c.dtype, f"{name} full rows")
+    fcols = np.array([0, c.N // 2 + 5, c.N - 1])
+    ref_c = oracle.gemm_epilogue_sampled(c.A, c.B, c.bias, c.M, c.N, c.K, c.dtype, c.act, np.arange(c.M), fcols)
+    H.check_tolerance(y[:, fcols], ref_c, c.dtype, f"{name} full columns")
+    assert np.isfinite(y).all()
+    # properties that hold at any size: ReLU output is non-negative; results are reproducible
+    if c.act == RELU:
+        assert (y >= 0).all()
+    bits2, _ = H.run_case(handle, c)
+    assert np.array_equal(bits, bits2)
+
+
+# ---------------------------------------------------------------- dispatcher, metamorphic relations, edge cases
+
+def test_dispatcher_choices(handle):
+    sel = handle.select_variant
+    assert sel(256, 256, 256, F32) == V.VARIANT_F32_TILED
+    assert sel(255, 255, 255, F32) == V.VARIANT_GENERIC
+    assert sel(1, 8192, 8192, BF16) in (V.VARIANT_GEMV_SPLITK, V.VARIANT_SKINNY_UMMA)
+    assert sel(16, 14336, 4096, BF16) == V.VARIANT_SKINNY_UMMA
+    assert sel(4096, 4096, 4096, BF16) == V.VARIANT_UMMA
+    assert sel(8192, 8192, 16384, BF16) == V.VARIANT_UMMA
+    assert sel(4096, 4100, 4096, BF16) == V.VARIANT_GENERIC      # N % 8 != 0
+    assert sel(0, 1, 1, BF16) == -1
+
+
+def test_unaligned_shapes_and_pointers_fall_back_to_the_generic_kernel(handle):
+    before = handle.launch_count()
+    parity(handle, synth.make_case("c4", M=130, N=262, K=100))       # N % 8 != 0
+    parity(handle, synth.make_case("c1", M=30, N=31, K=33))          # fp32, N % 4 != 0
+    assert handle.launch_count() == before + 2
+    # a 2-byte aligned (not 16-byte aligned) bf16 B pointer
+    c = synth.make_case("c4", M=128, N=256, K=64)
+    A = H.to_device(c.A, BF16, (c.M, c.K))
+    Bbuf = torch.zeros(c.K * c.N + 8, dtype=torch.bfloat16, device="cuda:0")
+    Bv = Bbuf[1:1 + c.K * c.N].view(c.K, c.N)
+    Bv.copy_(H.to_device(c.B, BF16, (c.K, c.N)))
+    bias = H.to_device(c.bias, BF16, (c.N,))
+    Y = torch.empty(c.M, c.N, dtype=torch.bfloat16, device="cuda:0")
+    rc = handle.gemm_epilogue_raw(A.data_ptr(), Bv.data_ptr(), bias.data_ptr(), Y.data_ptr(), c.M, c.N, c.K, BF16,
+                                  c.act, torch.cuda.current_stream().cuda_stream)
+    assert rc == binding.OK
+    torch.cuda.synchronize()
+    H.check_tolerance(oracle.widen(H.to_host_bits(Y, BF16), BF16), H.oracle_full(c), BF16, "unaligned B")
+
+
+def test_error_codes(handle):
+    x = torch.zeros(64, dtype=torch.float32, device="cuda:0")
+    p = x.data_ptr()
+    call = handle.gemm_epilogue_raw
+    assert call(None, p, None, p, 1, 1, 1, F32, NONE) == binding.ERR_INVALID_ARG
+    assert call(p, p, None, None, 1, 1, 1, F32, NONE) == binding.ERR_INVALID_ARG
+    assert call(p, p, None, p, 0, 1, 1, F32, NONE) == binding.ERR_INVALID_ARG
+    assert call(p, p, None, p, 1, -3, 1, F32, NONE) == binding.ERR_INVALID_ARG
+    assert call(p, p, None, p, 1, 1, 2 ** 31, F32, NONE) == binding.ERR_INVALID_ARG
+    assert call(p, p, None, p, 1, 1, 1, 7, NONE) == binding.ERR_INVALID_ARG
+    assert call(p, p, None, p, 1, 1, 1, F32, 9) == binding.ERR_INVALID_ARG
+    assert call(p + 2, p, None, p + 32, 1, 1, 1, F32, NONE) == binding.ERR_ALIGNMENT
+    assert call(p + 1, p, None, p + 32, 1, 1, 1, BF16, NONE) == binding.ERR_ALIGNMENT
+    handle.force_variant(V.VARIANT_UMMA)
+    assert call(p, p, None, p + 128, 2, 2, 2, F32, NONE) == binding.ERR_UNSUPPORTED
+    handle.force_variant(V.VARIANT_GEMV_SPLITK)
+    assert call(p, p, None, p + 128, 8, 8, 8, BF16, NONE) == binding.ERR_UNSUPPORTED     # M > 4
+    handle.force_variant(V.VARIANT_AUTO)
+    assert handle.get_last_status() == binding.OK
+    with pytest.raises(binding.OptimlError):
+        handle.force_variant(17)
+
+
+@pytest.mark.parametrize("variant,name,M,N,K", [(V.VARIANT_F32_TILED, "c1", 96, 128, 256),
+                                                (V.VARIANT_GEMV_SPLITK, "c2", 2, 1024, 2048),
+                                                (V.VARIANT_SKINNY_UMMA, "c3", 16, 1160, 1096),
+                                                (V.VARIANT_UMMA, "c4", 384, 512, 512)])
+def test_metamorphic_relations(handle, variant, name, M, N, K):
+    c = synth.make_case(name, M=M, N=N, K=K, act=RELU)
+    handle.force_variant(variant)
+    bits, y = H.run_case(handle, c)
+    bits_again, _ = H.run_case(handle, c)
+    assert np.array_equal(bits, bits_again), "same call, different bits"
+    # permuting the rows of A permutes the rows of Y, bit for bit
+    rp = np.random.default_rng(3).permutation(M)
+    cp = synth.Case(c.name, M, N, K, c.dtype, c.act, c.A.reshape(M, K)[rp].reshape(-1), c.B, c.bias)
+    bits_p, _ = H.run_case(handle, cp)
+    assert np.array_equal(bits_p.reshape(M, N), bits.reshape(M, N)[rp])
+    # scaling A and bias by 4 scales Y by 4 exactly (ReLU is positively homogeneous)
+    if c.dtype == F32:
+        c4 = synth.Case(c.name, M, N, K, c.dtype, c.act, c.A * np.float32(4), c.B, c.bias * np.float32(4))
+    else:
+        up = lambda b: np.where((b & 0x7FFF) == 0, b, b + np.uint16(2 << 7)).astype(np.uint16)   # exponent + 2
+        c4 = synth.Case(c.name, M, N, K, c.dtype, c.act, up(c.A), c.B, up(c.bias))
+    _, y4 = H.run_case(handle, c4)
+    assert np.array_equal(y4, 4.0 * y)
+
+
+def test_host_entry_point(handle):
+    c = synth.make_case("c4", M=256, N=512, K=320)
+    A = H.to_device(c.A, BF16, (c.M, c.K), "cpu").pin_memory()
+    B = H.to_device(c.B, BF16, (c.K, c.N), "cpu").pin_memory()
+    bias = H.to_device(c.bias, BF16, (c.N,), "cpu").pin_memory()
+    Y = torch.full((c.M, c.N), float("nan"), dtype=torch.bfloat16).pin_memory()
+    for _ in range(2):      # second call reuses the staging buffers
+        handle.gemm_epilogue_host(A, B, bias, Y, c.act)
+        H.check_tolerance(oracle.widen(H.to_host_bits(Y, BF16), BF16), H.oracle_full(c), BF16, "host entry point")
+
+
+def test_many_shapes_back_to_back_leave_the_scratch_clean(handle):
+    # split-K and stream-K kernels share arrival counters; interleave shapes and check all
+    cases = [synth.make_case("c3", M=16, N=1160, K=1096), synth.make_case("c2", M=1, N=2048, K=4096),
+             synth.make_case("c3", M=8, N=392, K=2056), synth.make_case("c2", M=3, N=520, K=1500)]
+    refs = [H.oracle_full(c) for c in cases]
+    for _ in range(3):
+        for c, r in zip(cases, refs):
+            _, y = H.run_case(handle, c)
+            H.check_tolerance(y, r, c.dtype, "interleaved")
