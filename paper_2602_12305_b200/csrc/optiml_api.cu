@@ -26,7 +26,7 @@ namespace {
 constexpr int kVersion = 10000 * 0 + 100 * 1 + 0;
 constexpr size_t kPartialBytes = (size_t)32 << 20;   // split-K / stream-K partial sums
 constexpr int kNumCounters = 1 << 16;                 // one arrival counter per column block / tile
-constexpr int kMapCache = 16;
+constexpr int kMapCache = 32;
 
 typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                     const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,

@@ -1,0 +1,73 @@
+"""Run one named workload a few times through the C ABI -- the command line used for
+profiling (ncu) and for quick timing of a forced variant.
+
+    python -m paper_2602_12305_b200.run_case --workload c3 [--variant auto|0..4] [--iters 3]
+        [--M m --N n --K k] [--sets 2] [--time]
+
+Each iteration uses the next of `--sets` distinct buffer sets.  With --time, CUDA-event
+times per launch are printed (median / min) with the implied TFLOP/s and GB/s.
+"""
+from __future__ import annotations
+
+import argparse
+import statistics
+
+import numpy as np
+import torch
+
+from . import binding, synth
+
+
+def _dev(arr, dtype, shape):
+    if dtype == synth.F32:
+        return torch.from_numpy(arr).view(*shape).cuda()
+    return torch.from_numpy(arr.view(np.int16)).view(torch.bfloat16).view(*shape).cuda()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="c2", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--variant", default="auto")
+    ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=1)
+    ap.add_argument("--sets", type=int, default=2)
+    ap.add_argument("--M", type=int)
+    ap.add_argument("--N", type=int)
+    ap.add_argument("--K", type=int)
+    ap.add_argument("--time", action="store_true")
+    a = ap.parse_args()
+
+    c = synth.make_case(a.workload, M=a.M, N=a.N, K=a.K)
+    h = binding.Handle(0)
+    if a.variant != "auto":
+        h.force_variant(int(a.variant))
+    tdt = torch.float32 if c.dtype == synth.F32 else torch.bfloat16
+    A0, B0, b0 = _dev(c.A, c.dtype, (c.M, c.K)), _dev(c.B, c.dtype, (c.K, c.N)), _dev(c.bias, c.dtype, (c.N,))
+    sets = [(A0, B0, b0, torch.empty((c.M, c.N), dtype=tdt, device="cuda"))]
+    for _ in range(a.sets - 1):
+        sets.append((A0.clone(), B0.clone(), b0.clone(), torch.empty((c.M, c.N), dtype=tdt, device="cuda")))
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(a.iters + 1)]
+    for i in range(a.warmup):
+        A, B, b, Y = sets[i % len(sets)]
+        h.gemm_epilogue(A, B, b, c.act, Y=Y)
+    torch.cuda.synchronize()
+    ev[0].record()
+    for i in range(a.iters):
+        A, B, b, Y = sets[(a.warmup + i) % len(sets)]
+        h.gemm_epilogue(A, B, b, c.act, Y=Y)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    status = h.get_last_status()
+    name = binding.variant_name(h.select_variant(c.M, c.N, c.K, c.dtype))
+    print(f"{a.workload} {c.M}x{c.N}x{c.K} via {name}: {a.iters} launches, status {binding.status_string(status)}")
+    if a.time:
+        ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(a.iters)]
+        med, mn = statistics.median(ms), min(ms)
+        print(f"  us per launch: median {med * 1e3:.2f}  min {mn * 1e3:.2f}   "
+              f"TFLOP/s {c.flops / 1e12 / (med / 1e3):.1f}   GB/s {c.algorithmic_bytes / 1e9 / (med / 1e3):.0f}")
+    h.destroy()
+    return 0 if status == binding.OK else 1
+
+
+if __name__ == "__main__":
+    raise SystemExit(main())
