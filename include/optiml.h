@@ -113,6 +113,44 @@ optiml_status_t optiml_gemm_epilogue_host(optiml_handle_t h, const void* A_host,
                                           optiml_dtype_t dtype, optiml_act_t act, void* stream);
 
 /*
+ * Y = act(A . B + bias) for bf16 GEMV-like problems, for callers that must not allocate.
+ * (The paper has no counterpart of this entry point; the operation is the one defined at
+ * the top of this header.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off the table -- a process whose
+ * device memory has been handed in full to another allocator (an inference server's
+ * arena, a framework's caching allocator) so that a fresh cudaMalloc fails, or a
+ * latency-critical loop that cannot afford the device-wide synchronisation an allocation
+ * may imply.  Such callers cannot create a handle either, because optiml_create
+ * allocates the handle's scratch.  This call takes no handle and calls no cudaMalloc,
+ * cudaFree or other allocating routine; the split-K scratch it needs (arrival counters
+ * and partial sums, 2 MiB + 1 KiB) is a fixed array inside the library image, which every
+ * GPU that loads the library holds until the process exits.
+ *
+ *   A, B, bias, Y   device pointers as for optiml_gemm_epilogue, dtype bf16, 16-byte
+ *                   aligned; bias may be NULL; the caller owns all four
+ *   M               1..4
+ *   N               multiple of 8, at most 65536 (the fixed scratch covers no more)
+ *   K               >= 1
+ *   device          CUDA device that owns the pointers and `stream`
+ *   stream          cudaStream_t (NULL = default stream); work is enqueued, not awaited
+ *
+ * Returns OPTIML_ERR_UNSUPPORTED for M > 4, N > 65536 or N % 8 != 0 (nothing is
+ * launched), ALIGNMENT for pointers that are not 16-byte aligned, ARCH on a device that
+ * is not compute capability 10.0, INVALID_ARG / CUDA as elsewhere.
+ *
+ * The first call on each device looks up the scratch array's device address and the SM
+ * count (host-side queries only) and keeps them for later calls; that first call
+ * should come before any stream capture.  Every call on a device shares the one array, which still
+ * holds what the previous call left: each call re-zeroes the counters on `stream` before
+ * its kernel.  Two calls whose work overlaps on the GPU (different streams, or different
+ * host threads) therefore race on the scratch and give undefined results -- keep calls on
+ * one device in a single stream order.  Not thread-safe on first use per device.
+ */
+optiml_status_t optiml_gemv_noalloc(const void* A, const void* B, const void* bias, void* Y, int64_t M, int64_t N,
+                                    int64_t K, optiml_act_t act, int device, void* stream);
+
+/*
  * Read the device-written status word (synchronises the device): OPTIML_OK, or
  * OPTIML_ERR_TIMEOUT if any kernel of this handle gave up a bounded wait since the
  * last call of this function; the word is cleared.  A call that reported a

@@ -28,6 +28,7 @@ EXPORTS = {
     "optiml_destroy": (_ci, [_vp]),
     "optiml_gemm_epilogue": (_ci, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _ci, _vp]),
     "optiml_gemm_epilogue_host": (_ci, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _ci, _vp]),
+    "optiml_gemv_noalloc": (_ci, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _ci, _vp]),
     "optiml_get_last_status": (_ci, [_vp]),
     "optiml_force_variant": (_ci, [_vp, _ci]),
     "optiml_select_variant": (_ci, [_vp, _i64, _i64, _i64, _ci]),
@@ -85,6 +86,28 @@ def _dtype_code(t: torch.Tensor) -> int:
     if t.dtype == torch.bfloat16:
         return BF16
     raise TypeError(f"unsupported dtype {t.dtype}: float32 or bfloat16 only")
+
+
+def gemv_noalloc_raw(A: int, B: int, bias: int | None, Y: int, M: int, N: int, K: int, act: int, device: int = 0,
+                     stream: int | None = None) -> int:
+    """optiml_gemv_noalloc with raw device addresses; returns the status code."""
+    return load_library().optiml_gemv_noalloc(A, B, bias, Y, M, N, K, act, device, stream)
+
+
+def gemv_noalloc(A: torch.Tensor, B: torch.Tensor, bias: torch.Tensor | None, Y: torch.Tensor, act: int,
+                 stream: torch.cuda.Stream | None = None) -> torch.Tensor:
+    """Y = act(A @ B + bias) for bf16, M <= 4, N <= 65536, without a handle and without any
+    allocation inside the library (its scratch is a fixed array in the library image).
+    For callers whose device memory is owned by another allocator or who cannot afford an
+    allocation's synchronisation.  The caller provides Y.  Calls on one device share the
+    scratch: keep them in one stream order."""
+    M, K = A.shape
+    N = B.shape[1]
+    dev = A.device.index
+    st = (stream or torch.cuda.current_stream(dev)).cuda_stream
+    _check(gemv_noalloc_raw(A.data_ptr(), B.data_ptr(), None if bias is None else bias.data_ptr(), Y.data_ptr(),
+                            M, N, K, act, dev, st), "optiml_gemv_noalloc")
+    return Y
 
 
 class Handle:

@@ -485,4 +485,78 @@ const char* optiml_variant_name(int variant) {
 
 int optiml_version(void) { return kVersion; }
 
+// ---------------------------------------------------------------- entry point that allocates nothing
+
+}  // extern "C"
+
+namespace {
+
+// Scratch of optiml_gemv_noalloc: arrival counters (one per 256-column block) followed by the
+// split-K partial sums.  It lives in the library image, so every GPU that loads the library
+// holds these bytes until the process exits, whether or not the entry point is ever called.
+constexpr int kNoAllocMaxN = 65536;
+constexpr size_t kNoAllocCounterBytes = (kNoAllocMaxN / kGemvCols) * sizeof(unsigned int);   // 1 KiB
+constexpr size_t kNoAllocPartialBytes = (size_t)2 << 20;                                      // 2 MiB
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocCounterBytes + kNoAllocPartialBytes];
+
+constexpr int kNoAllocMaxDevices = 64;
+unsigned char* g_noalloc_ptr[kNoAllocMaxDevices] = {};   // device address of the array, per device
+int g_noalloc_sms[kNoAllocMaxDevices] = {};
+
+}  // namespace
+
+extern "C" {
+
+optiml_status_t optiml_gemv_noalloc(const void* A, const void* B, const void* bias, void* Y, int64_t M, int64_t N,
+                                    int64_t K, optiml_act_t act, int device, void* stream) {
+    if (!A || !B || !Y || M < 1 || N < 1 || K < 1 || K > INT32_MAX) return OPTIML_ERR_INVALID_ARG;
+    if (act != OPTIML_ACT_NONE && act != OPTIML_ACT_RELU && act != OPTIML_ACT_GELU_TANH) return OPTIML_ERR_INVALID_ARG;
+    if (device < 0 || device >= kNoAllocMaxDevices) return OPTIML_ERR_INVALID_ARG;
+    // limits of the fixed scratch and of the kernel: refuse, never truncate
+    if (M > 4 || N > kNoAllocMaxN || N % 8 != 0) return OPTIML_ERR_UNSUPPORTED;
+    if (!(aligned16(A) && aligned16(B) && aligned16(bias) && aligned16(Y))) return OPTIML_ERR_ALIGNMENT;
+
+    DeviceGuard guard(device);
+    if (!g_noalloc_ptr[device]) {
+        // One-time set-up on this device (it must be the current one here).  In host code the
+        // name of a __device__ array is only a stand-in; the address a kernel may use comes
+        // from cudaGetSymbolAddress.
+        int major = 0, minor = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+            cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, device) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+            return OPTIML_ERR_CUDA;
+        if (major != 10 || minor != 0) return OPTIML_ERR_ARCH;
+        unsigned char* p = nullptr;
+        if (cudaGetSymbolAddress((void**)&p, g_noalloc_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return OPTIML_ERR_CUDA;
+        }
+        g_noalloc_sms[device] = sms;
+        g_noalloc_ptr[device] = p;
+    }
+    unsigned char* base = g_noalloc_ptr[device];
+    unsigned int* counters = reinterpret_cast<unsigned int*>(base);
+    float* partials = reinterpret_cast<float*>(base + kNoAllocCounterBytes);
+
+    const int m = (int)M, n = (int)N, k = (int)K;
+    const int MR = m == 1 ? 1 : (m == 2 ? 2 : 4);
+    const int64_t col_blocks = ceil_div64(N, kGemvCols);
+    int64_t S = (2 * (int64_t)g_noalloc_sms[device]) / col_blocks;
+    if (S > K / 64) S = K / 64;
+    const int64_t per_slice = (int64_t)MR * kGemvCols * sizeof(float);
+    if (S * col_blocks * per_slice > (int64_t)kNoAllocPartialBytes) S = kNoAllocPartialBytes / (col_blocks * per_slice);
+    if (S < 1) S = 1;
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // The array keeps whatever the last call left behind.  The counters must start at zero
+    // (the partial sums need not: every slot that is read is written first).
+    if (cudaMemsetAsync(counters, 0, kNoAllocCounterBytes, st) != cudaSuccess) return OPTIML_ERR_CUDA;
+    dim3 grid((unsigned)col_blocks, (unsigned)S);
+    if (MR == 1) launch_gemv_mr<1>(A, B, bias, Y, m, n, k, (int)act, grid, partials, counters, st);
+    else if (MR == 2) launch_gemv_mr<2>(A, B, bias, Y, m, n, k, (int)act, grid, partials, counters, st);
+    else launch_gemv_mr<4>(A, B, bias, Y, m, n, k, (int)act, grid, partials, counters, st);
+    return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
 }  // extern "C"
