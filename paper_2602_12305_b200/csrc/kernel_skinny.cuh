@@ -6,18 +6,32 @@
 //   MMA "A" operand = a 128(n) x 64(k) tile of B, N contiguous (MN-major), two 64-column
 //                     TMA boxes with 128-byte swizzle;
 //   MMA "B" operand = the MP x 64 tile of A (rows >= M are zero-filled by TMA), K-major;
-//   accumulator     = 128 TMEM lanes (n) x MP fp32 columns (m), double buffered.
+//   accumulator     = 128 TMEM lanes (n) x MP fp32 columns (m) per column tile.
 //
-// Work is cut stream-K style: the (column tile, K block) units, in column-tile-major
-// order, are dealt in equal contiguous ranges to one CTA per SM, so every SM streams the
-// same number of bytes whatever N and K are.  A CTA's range is a sequence of segments
-// (one column tile, a range of K blocks).  A segment spanning all of K goes straight
-// through the fused epilogue.  Otherwise the fp32 partial tile is written to the handle's
-// scratch and an arrival counter per column tile is bumped; the CTA that arrives last
-// (nobody waits) adds the partials in K order, applies bias + activation and stores Y.
+// Schedule (SkinnyPlan, made on the host).  One CTA per SM.  The (column tile, K block)
+// grid, T x KB units, is cut into one rectangle per CTA, all of about the same area, so
+// every SM streams the same number of bytes.  The rectangles are arranged in horizontal
+// BANDS: a band is a range of K blocks in which the T column tiles are dealt left to
+// right to the band's CTAs.  A CTA sweeps its rectangle K-major (for each K block, all of
+// its column tiles) with one TMEM accumulator per column tile.  All CTAs of a band
+// therefore walk down the same rows of B at the same pace and between them read whole
+// rows: DRAM sees long sequential bursts.  (CTAs streaming unrelated 256-byte wide strips
+// reach only half the HBM throughput on B200.)
+//   * S "full" bands: T CTAs each, one column tile per CTA;
+//   * up to two "wide" bands for the CTAs left over (or for all CTAs when T > CTAs), where
+//     a CTA takes several adjacent column tiles; the band heights are chosen so that all
+//     rectangles have the same area.
+//
+// With a single band every column tile is finished by one CTA and goes straight through
+// the fused epilogue.  Otherwise each band's CTA writes its fp32 partial tile to the
+// handle's scratch and bumps the tile's arrival counter; the CTA that arrives last (nobody
+// waits) adds the partials in band (= K) order, applies bias + activation and stores Y.
 // The order of the sum is fixed, so results are reproducible.
 //
-// Roles: warp 0 TMA producer, warp 1 TMEM allocation + MMA issue, warps 2-5 epilogue.
+// Roles: warp 0 TMA producer (a ring of B tiles, a small ring of A tiles: one A tile per
+// K block serves all the column tiles of the sweep), warp 1 TMEM allocation + MMA issue,
+// warps 2-5 epilogue.  TMEM holds two sets of accumulators so that, when a CTA's
+// rectangle is wider than one set, the epilogue of one chunk overlaps the next sweep.
 // All mbarrier waits are bounded; see kernel_umma.cuh for the tear-down protocol.
 #pragma once
 
@@ -29,18 +43,27 @@ namespace optiml {
 template <int MP>
 struct SkinnyCfg {
     static_assert(MP == 16 || MP == 32 || MP == 64 || MP == 128, "padded M");
-    static constexpr int BN = 128, BK = 64;
-    static constexpr int kBChunkBytes = BK * 64 * 2;           // 64 k-rows x 64 columns: 8 KiB
-    static constexpr int kBBytes = 2 * kBChunkBytes;           // 16 KiB
-    static constexpr int kABytes = MP * BK * 2;
-    static constexpr int kStageBytes = kBBytes + kABytes;      // multiple of 1024
-    static constexpr int kMaxStages = 12;
-    static constexpr int kFit = (216 * 1024) / kStageBytes;
-    static constexpr int kStages = kFit < kMaxStages ? kFit : kMaxStages;
+    // One pipeline stage carries kSub sub-blocks of 64 K rows: every stage costs one
+    // tcgen05.commit / mbarrier round trip, and with the tiny MMAs of this kernel that round
+    // trip, not HBM, limits a 64-row stage.
+    static constexpr int kSub = 2;
+    static constexpr int BN = 128, BK = 64 * kSub;
+    static constexpr int kBChunkBytes = 64 * 64 * 2;           // 64 k-rows x 64 columns: 8 KiB
+    static constexpr int kBSubBytes = 2 * kBChunkBytes;        // 64 k-rows x 128 columns
+    static constexpr int kBBytes = kSub * kBSubBytes;          // one stage of the B ring
+    static constexpr int kASubBytes = MP * 64 * 2;
+    static constexpr int kABytes = kSub * kASubBytes;          // one slot of the A ring
+    static constexpr int kFit = (212 * 1024 - kABytes) / (kBBytes + kABytes);
+    static constexpr int kStages = kFit < 12 ? kFit : 12;
+    // The A ring needs no "empty" barrier: a slot is reused kAStages K blocks later, and by
+    // then the producer has waited for B stages whose release implies that every MMA of the
+    // old K block is done (it can be at most kStages stages ahead of the MMAs).
+    static constexpr int kAStages = kStages + 1;
     static constexpr int kThreads = 192;
-    static constexpr int kTmemCols = 2 * MP < 32 ? 32 : 2 * MP;
+    static constexpr int kAcc = 256 / MP < 8 ? 256 / MP : 8;   // column tiles per sweep
+    static constexpr int kTmemCols = 2 * kAcc * MP;            // 256 (MP = 16) or 512
     static constexpr int kChunk = MP < 32 ? MP : 32;           // accumulator columns per tcgen05.ld
-    static constexpr int kSmemBytes = kStages * kStageBytes + 512 + 1024;
+    static constexpr int kSmemBytes = kStages * kBBytes + kAStages * kABytes + 512 + 1024;
     static constexpr int kSlotFloats = MP * BN;                // one partial tile in scratch
 };
 
@@ -48,17 +71,134 @@ template <int MP>
 struct SkinnyShared {
     uint64_t full[SkinnyCfg<MP>::kStages];
     uint64_t empty[SkinnyCfg<MP>::kStages];
+    uint64_t a_full[SkinnyCfg<MP>::kAStages];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint64_t drain;
     uint32_t tmem_base;
     volatile int abort;
-    int last_flag;
+    int last_flag[8];
+    int vote[4];
 };
 
-// Stream-K bookkeeping: U units over G CTAs; CTA c owns units [U*c/G, U*(c+1)/G).
-__device__ __forceinline__ int64_t sk_begin(int64_t U, int G, int c) { return U * c / G; }
-__device__ __forceinline__ int sk_owner(int64_t U, int G, int64_t u) { return (int)(((u + 1) * G + U - 1) / U - 1); }
+// Host-made schedule; see the header comment.
+struct SkinnyPlan {
+    int T;         // column tiles
+    int KB;        // K blocks
+    int G;         // CTAs = S*T + G1 + G2
+    int S;         // full bands, covering K blocks [0, k_split)
+    int k_split;
+    int G1;        // CTAs of wide band 1, K blocks [k_split, k_mid)
+    int k_mid;
+    int G2;        // CTAs of wide band 2, K blocks [k_mid, KB)
+    int nbands;    // S + (G1 > 0) + (G2 > 0): segments per column tile
+};
+
+struct SkinnyRect {
+    int t0, t1, kb0, kb1, band;
+};
+
+__host__ __device__ __forceinline__ SkinnyRect skinny_rect(const SkinnyPlan& p, int c) {
+    SkinnyRect r;
+    if (c < p.S * p.T) {
+        const int s = c / p.T;
+        r.t0 = c % p.T;
+        r.t1 = r.t0 + 1;
+        r.kb0 = (int)((int64_t)p.k_split * s / p.S);
+        r.kb1 = (int)((int64_t)p.k_split * (s + 1) / p.S);
+        r.band = s;
+        return r;
+    }
+    int i = c - p.S * p.T;
+    if (i < p.G1) {
+        r.t0 = (int)((int64_t)p.T * i / p.G1);
+        r.t1 = (int)((int64_t)p.T * (i + 1) / p.G1);
+        r.kb0 = p.k_split;
+        r.kb1 = p.k_mid;
+        r.band = p.S;
+    } else {
+        i -= p.G1;
+        r.t0 = (int)((int64_t)p.T * i / p.G2);
+        r.t1 = (int)((int64_t)p.T * (i + 1) / p.G2);
+        r.kb0 = p.k_mid;
+        r.kb1 = p.KB;
+        r.band = p.S + (p.G1 > 0 ? 1 : 0);
+    }
+    return r;
+}
+
+// Best balanced banding for `num_sms` CTAs.  cost = the largest rectangle area (K blocks
+// x column tiles) any CTA has to stream; ties go to fewer bands (fewer partial tiles).
+// `max_slots` bounds bands * T, the partial tiles the scratch can hold.
+inline SkinnyPlan make_skinny_plan(int64_t tiles, int64_t kblocks, int num_sms, int64_t max_slots) {
+    const int64_t T = tiles, KB = kblocks;
+    SkinnyPlan best;
+    best.T = (int)T;
+    best.KB = (int)KB;
+    // fallback: one wide band over everything
+    best.S = 0;
+    best.k_split = 0;
+    best.G1 = (int)(T < num_sms ? T : num_sms);
+    best.k_mid = (int)KB;
+    best.G2 = 0;
+    best.nbands = 1;
+    best.G = best.G1;
+    int64_t best_cost = ((T + best.G1 - 1) / best.G1) * KB;
+
+    auto consider = [&](int S, int64_t k_split, int G1, int64_t k_mid, int G2) {
+        const int nb = S + (G1 > 0) + (G2 > 0);
+        if (nb < 1 || (nb > 1 && nb * T > max_slots)) return;
+        if (S > 0 && k_split < S) return;
+        if (G1 > 0 && k_mid <= k_split) return;
+        if (G2 > 0 && KB <= k_mid) return;
+        if (G2 == 0 && k_mid != KB) return;
+        if (G1 == 0 && (k_split != KB || G2 != 0)) return;
+        int64_t cost = S > 0 ? (k_split + S - 1) / S : 0;
+        if (G1 > 0) {
+            const int64_t c1 = ((T + G1 - 1) / G1) * (k_mid - k_split);
+            if (c1 > cost) cost = c1;
+        }
+        if (G2 > 0) {
+            const int64_t c2 = ((T + G2 - 1) / G2) * (KB - k_mid);
+            if (c2 > cost) cost = c2;
+        }
+        if (cost < best_cost || (cost == best_cost && nb < best.nbands)) {
+            best_cost = cost;
+            best.S = S;
+            best.k_split = (int)k_split;
+            best.G1 = G1;
+            best.k_mid = (int)k_mid;
+            best.G2 = G2;
+            best.nbands = nb;
+            best.G = (int)(S * T) + G1 + G2;
+        }
+    };
+
+    const int s_max = (int)(num_sms / T);
+    for (int S = s_max; S >= 1; --S) {
+        const int left = (int)(num_sms - S * T);
+        consider(S, KB, 0, KB, 0);                               // full bands only
+        if (left > 0) {
+            const int G1 = (int)(left < T ? left : T);
+            const int64_t w1 = (T + G1 - 1) / G1;
+            // S*a + h = KB with a ~ w1*h
+            const int64_t h0 = KB / (S * w1 + 1);
+            for (int64_t h = h0 - 1; h <= h0 + 2; ++h)
+                if (h >= 1 && h < KB) consider(S, KB - h, G1, KB, 0);
+        }
+    }
+    // no full band: two wide bands over all CTAs (covers T >= CTAs as well)
+    for (int G1 = 1; G1 < num_sms; ++G1) {
+        if (G1 > T) break;
+        int G2 = num_sms - G1;
+        if (G2 > T) G2 = (int)T;
+        const int64_t w1 = (T + G1 - 1) / G1, w2 = (T + G2 - 1) / G2;
+        const int64_t h0 = KB * w2 / (w1 + w2);
+        for (int64_t h = h0 - 1; h <= h0 + 2; ++h)
+            if (h >= 1 && h < KB) consider(0, 0, G1, h, G2);
+    }
+    return best;
+}
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
@@ -66,35 +206,33 @@ template <int MP>
 __global__ void __launch_bounds__(SkinnyCfg<MP>::kThreads, 1)
 gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                         const __nv_bfloat16* __restrict__ bias, __nv_bfloat16* __restrict__ Y, int M, int N, int K,
-                        int act, float* __restrict__ partials, unsigned int* __restrict__ counters,
-                        int* __restrict__ status) {
+                        int act, const __grid_constant__ SkinnyPlan plan, float* __restrict__ partials,
+                        unsigned int* __restrict__ counters, int* __restrict__ status) {
     using C = SkinnyCfg<MP>;
     using Sh = SkinnyShared<MP>;
     static_assert(sizeof(Sh) <= 512, "barrier block");
     extern __shared__ uint8_t smem_raw[];
     Sh* sh = reinterpret_cast<Sh*>(smem_raw);
-    const uint32_t ring_base = (ptx::smem_u32(smem_raw) + 512 + 1023) & ~1023u;
+    const uint32_t ring_base = (ptx::smem_u32(smem_raw) + 512 + 1023) & ~1023u;     // B ring, then A ring
     uint8_t* ring = smem_raw + (ring_base - ptx::smem_u32(smem_raw));
+    const uint32_t aring_base = ring_base + C::kStages * C::kBBytes;
+    uint8_t* aring = ring + C::kStages * C::kBBytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int G = gridDim.x, c = blockIdx.x;
-    const int KB = (K + C::BK - 1) / C::BK;
-    const int tiles_n = (N + C::BN - 1) / C::BN;
-    const int64_t U = (int64_t)tiles_n * KB;
-    const int64_t u0 = sk_begin(U, G, c), u1 = sk_begin(U, G, c + 1);
+    const SkinnyRect rect = skinny_rect(plan, blockIdx.x);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::kStages; ++s) {
             ptx::mbar_init(&sh->full[s], 1);
             ptx::mbar_init(&sh->empty[s], 1);
         }
+        for (int s = 0; s < C::kAStages; ++s) ptx::mbar_init(&sh->a_full[s], 1);
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(&sh->tmem_full[a], 1);
             ptx::mbar_init(&sh->tmem_empty[a], 128);
         }
         ptx::mbar_init(&sh->drain, 1);
         sh->abort = 0;
-        sh->last_flag = 0;
         ptx::fence_mbar_init();
     }
     if (warp == 1) {
@@ -113,28 +251,45 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             ptx::prefetch_tensormap(&map_b);
             const uint64_t pol_stream = ptx::policy_evict_first();   // B is read exactly once
             const uint64_t pol_keep = ptx::policy_evict_last();      // A is re-read by every CTA
-            uint32_t it = 0;
+            uint32_t it = 0, ait = 0;
             bool ok = true;
-            for (int64_t u = u0; u < u1; ++u, ++it) {
-                const int tile = (int)(u / KB), kb = (int)(u % KB);
-                const int s = it % C::kStages;
-                const uint32_t ph = (it / C::kStages) & 1;
-                if (sh->abort || !ptx::mbar_wait(&sh->empty[s], ph ^ 1)) { ok = false; break; }
-                uint8_t* b_dst = ring + s * C::kStageBytes;
-                uint8_t* a_dst = b_dst + C::kBBytes;
-                ptx::mbar_arrive_expect_tx(&sh->full[s], C::kStageBytes);
-                ptx::tma_load_2d_hint(b_dst, &map_b, &sh->full[s], tile * C::BN, kb * C::BK, pol_stream);
-                ptx::tma_load_2d_hint(b_dst + C::kBChunkBytes, &map_b, &sh->full[s], tile * C::BN + 64, kb * C::BK,
-                                      pol_stream);
-                ptx::tma_load_2d_hint(a_dst, &map_a, &sh->full[s], kb * C::BK, 0, pol_keep);
+            for (int tc = rect.t0; tc < rect.t1 && ok; tc += C::kAcc) {
+                const int nt = min(C::kAcc, rect.t1 - tc);
+                for (int kb = rect.kb0; kb < rect.kb1 && ok; ++kb, ++ait) {
+                    const int sa = ait % C::kAStages;
+                    ptx::mbar_arrive_expect_tx(&sh->a_full[sa], C::kABytes);
+#pragma unroll
+                    for (int u = 0; u < C::kSub; ++u)
+                        ptx::tma_load_2d_hint(aring + sa * C::kABytes + u * C::kASubBytes, &map_a, &sh->a_full[sa],
+                                              kb * C::BK + u * 64, 0, pol_keep);
+                    for (int j = 0; j < nt; ++j, ++it) {
+                        const int s = it % C::kStages;
+                        if (sh->abort || !ptx::mbar_wait(&sh->empty[s], ((it / C::kStages) & 1) ^ 1)) { ok = false; break; }
+                        uint8_t* b_dst = ring + s * C::kBBytes;
+                        ptx::mbar_arrive_expect_tx(&sh->full[s], C::kBBytes);
+#pragma unroll
+                        for (int u = 0; u < C::kSub; ++u) {
+                            ptx::tma_load_2d_hint(b_dst + u * C::kBSubBytes, &map_b, &sh->full[s], (tc + j) * C::BN,
+                                                  kb * C::BK + u * 64, pol_stream);
+                            ptx::tma_load_2d_hint(b_dst + u * C::kBSubBytes + C::kBChunkBytes, &map_b, &sh->full[s],
+                                                  (tc + j) * C::BN + 64, kb * C::BK + u * 64, pol_stream);
+                        }
+                    }
+                }
             }
             if (!ok) {
                 atomicExch(status, kDevTimeout);
                 sh->abort = 1;
+                // copies already issued must land before the CTA may exit
                 const uint32_t n_back = it < (uint32_t)C::kStages ? it : (uint32_t)C::kStages;
                 for (uint32_t b = 1; b <= n_back; ++b) {
                     const uint32_t j = it - b;
                     ptx::mbar_wait(&sh->full[j % C::kStages], (j / C::kStages) & 1);
+                }
+                const uint32_t a_back = ait < (uint32_t)C::kAStages ? ait : (uint32_t)C::kAStages;
+                for (uint32_t b = 1; b <= a_back; ++b) {
+                    const uint32_t j = ait - b;
+                    ptx::mbar_wait(&sh->a_full[j % C::kAStages], (j / C::kAStages) & 1);
                 }
             }
         }
@@ -142,34 +297,35 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = ptx::umma_idesc_bf16(C::BN, MP, /*a_mn_major=*/true, /*b_mn_major=*/false);
-            uint32_t it = 0, seg_it = 0;
+            uint32_t it = 0, ait = 0, chunk_it = 0;
             bool ok = true;
-            for (int64_t u = u0; u < u1 && ok; ++seg_it) {
-                const int kb0 = (int)(u % KB);
-                const int64_t left = u1 - u;
-                const int kb1 = (int)(left < KB - kb0 ? kb0 + left : KB);
-                const int a = seg_it & 1;
-                const uint32_t aph = (seg_it >> 1) & 1;
-                if (sh->abort || !ptx::mbar_wait(&sh->tmem_empty[a], aph ^ 1)) { ok = false; break; }
+            for (int tc = rect.t0; tc < rect.t1 && ok; tc += C::kAcc, ++chunk_it) {
+                const int nt = min(C::kAcc, rect.t1 - tc);
+                const int half = chunk_it & 1;
+                if (sh->abort || !ptx::mbar_wait(&sh->tmem_empty[half], ((chunk_it >> 1) & 1) ^ 1)) { ok = false; break; }
                 ptx::tcgen05_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + a * MP;
-                for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                    const int s = it % C::kStages;
-                    const uint32_t ph = (it / C::kStages) & 1;
-                    if (sh->abort || !ptx::mbar_wait(&sh->full[s], ph)) { ok = false; break; }
-                    ptx::tcgen05_fence_after_sync();
-                    const uint32_t b_addr = ring_base + s * C::kStageBytes;   // tile of B
-                    const uint32_t a_addr = b_addr + C::kBBytes;              // tile of A
+                for (int kb = rect.kb0; kb < rect.kb1 && ok; ++kb, ++ait) {
+                    const int sa = ait % C::kAStages;
+                    if (sh->abort || !ptx::mbar_wait(&sh->a_full[sa], (ait / C::kAStages) & 1)) { ok = false; break; }
+                    const uint32_t a_addr = aring_base + sa * C::kABytes;            // tile of A
+                    for (int j = 0; j < nt; ++j, ++it) {
+                        const int s = it % C::kStages;
+                        if (sh->abort || !ptx::mbar_wait(&sh->full[s], (it / C::kStages) & 1)) { ok = false; break; }
+                        ptx::tcgen05_fence_after_sync();
+                        const uint32_t b_addr = ring_base + s * C::kBBytes;          // tile of B
+                        const uint32_t d_tmem = tmem_base + (half * C::kAcc + j) * MP;
 #pragma unroll
-                    for (int k4 = 0; k4 < C::BK / 16; ++k4) {
-                        const uint64_t da = ptx::umma_smem_desc(b_addr + k4 * 2048, C::kBChunkBytes, 1024);
-                        const uint64_t db = ptx::umma_smem_desc(a_addr + k4 * 32, 16, 1024);
-                        ptx::umma_bf16(d_tmem, da, db, idesc, (kb != kb0) || (k4 != 0));
+                        for (int k4 = 0; k4 < C::BK / 16; ++k4) {
+                            const uint64_t da = ptx::umma_smem_desc(b_addr + (k4 / 4) * C::kBSubBytes + (k4 % 4) * 2048,
+                                                                    C::kBChunkBytes, 1024);
+                            const uint64_t db = ptx::umma_smem_desc(a_addr + (k4 / 4) * C::kASubBytes + (k4 % 4) * 32,
+                                                                    16, 1024);
+                            ptx::umma_bf16(d_tmem, da, db, idesc, (kb != rect.kb0) || (k4 != 0));
+                        }
+                        ptx::umma_commit(&sh->empty[s]);
                     }
-                    ptx::umma_commit(&sh->empty[s]);
                 }
-                if (ok) ptx::umma_commit(&sh->tmem_full[a]);
-                u += kb1 - kb0;
+                if (ok) ptx::umma_commit(&sh->tmem_full[half]);
             }
             if (!ok) {
                 atomicExch(status, kDevTimeout);
@@ -184,74 +340,95 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         const int r = q * 32 + lane;                      // n within the column tile = TMEM lane
         const int et = threadIdx.x - 64;                  // 0..127 among the epilogue threads
         const int m_valid = M < MP ? M : MP;
-        uint32_t seg_it = 0;
+        const bool whole = plan.nbands == 1;
+        uint32_t chunk_it = 0;
         bool ok = true;
-        for (int64_t u = u0; u < u1 && ok; ++seg_it) {
-            const int tile = (int)(u / KB), kb0 = (int)(u % KB);
-            const int64_t left = u1 - u;
-            const int kb1 = (int)(left < KB - kb0 ? kb0 + left : KB);
-            const bool whole = (kb0 == 0 && kb1 == KB);
-            const int a = seg_it & 1;
-            const uint32_t aph = (seg_it >> 1) & 1;
-            bool got = !sh->abort && ptx::mbar_wait(&sh->tmem_full[a], aph);
+        for (int tc = rect.t0; tc < rect.t1 && ok; tc += C::kAcc, ++chunk_it) {
+            const int nt = min(C::kAcc, rect.t1 - tc);
+            const int half = chunk_it & 1;
+            bool got = !sh->abort && ptx::mbar_wait(&sh->tmem_full[half], (chunk_it >> 1) & 1);
             got = __all_sync(0xffffffffu, got);
+            // the four epilogue warps meet at named barriers below: they must take the same
+            // decision, so they vote (every warp reaches this barrier: its wait is bounded)
+            if (lane == 0) sh->vote[q] = got;
+            epi_bar_sync();
+            got = sh->vote[0] && sh->vote[1] && sh->vote[2] && sh->vote[3];
+            epi_bar_sync();
             if (!got) { ok = false; break; }
             ptx::tcgen05_fence_after_sync();
 
-            const int64_t n = (int64_t)tile * C::BN + r;
-            const float bv = (bias && n < N) ? __bfloat162float(bias[n]) : 0.0f;
-            float* slot = partials + ((size_t)2 * c + (u == u0 ? 0 : 1)) * C::kSlotFloats;
+            for (int j = 0; j < nt; ++j) {
+                const int tile = tc + j;
+                const int64_t n = (int64_t)tile * C::BN + r;
+                const float bv = (whole && bias && n < N) ? __bfloat162float(bias[n]) : 0.0f;
+                float* slot = partials + ((size_t)rect.band * plan.T + tile) * C::kSlotFloats;
 #pragma unroll 1
-            for (int m0 = 0; m0 < MP; m0 += C::kChunk) {
-                uint32_t v[C::kChunk];
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + a * MP + m0;
-                if constexpr (C::kChunk == 16) ptx::tmem_ld_32x16(taddr, v);
-                else ptx::tmem_ld_32x32(taddr, v);
-                ptx::tmem_ld_wait();
-                if (whole) {
+                for (int m0 = 0; m0 < MP; m0 += C::kChunk) {
+                    uint32_t v[C::kChunk];
+                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (half * C::kAcc + j) * MP + m0;
+                    if constexpr (C::kChunk == 16) ptx::tmem_ld_32x16(taddr, v);
+                    else ptx::tmem_ld_32x32(taddr, v);
+                    ptx::tmem_ld_wait();
+                    if (whole) {
 #pragma unroll
-                    for (int j = 0; j < C::kChunk; ++j) {
-                        const int m = m0 + j;
-                        if (m < m_valid && n < N)
-                            Y[(int64_t)m * N + n] = __float2bfloat16_rn(epilogue_rt<true>(__uint_as_float(v[j]), bv, act));
+                        for (int i = 0; i < C::kChunk; ++i) {
+                            const int m = m0 + i;
+                            if (m < m_valid && n < N)
+                                Y[(int64_t)m * N + n] =
+                                    __float2bfloat16_rn(epilogue_rt<true>(__uint_as_float(v[i]), bv, act));
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < C::kChunk; ++i)
+                            if (m0 + i < m_valid) slot[(m0 + i) * C::BN + r] = __uint_as_float(v[i]);
                     }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < C::kChunk; ++j)
-                        if (m0 + j < m_valid) slot[(m0 + j) * C::BN + r] = __uint_as_float(v[j]);
                 }
             }
-            // accumulator read out: hand it back before the (slower) cross-CTA part
+            // accumulators read out: hand them back before the (slower) cross-CTA part
             ptx::tcgen05_fence_before_sync();
-            ptx::mbar_arrive(&sh->tmem_empty[a]);
+            ptx::mbar_arrive(&sh->tmem_empty[half]);
 
             if (!whole) {
                 __threadfence();
                 epi_bar_sync();
-                const int64_t tile_first = (int64_t)tile * KB, tile_last = tile_first + KB - 1;
-                const int c_first = sk_owner(U, G, tile_first), c_last = sk_owner(U, G, tile_last);
-                if (et == 0) {
+                if (et < nt) {
+                    const int tile = tc + et;
                     const unsigned int prev = atomicAdd(&counters[tile], 1u);
-                    const int last = (prev == (unsigned int)(c_last - c_first));
-                    if (last) counters[tile] = 0u;        // everyone has arrived: re-arm for the next call
-                    sh->last_flag = last;
+                    const int last = (prev == (unsigned int)(plan.nbands - 1));
+                    if (last) counters[tile] = 0u;        // every band has arrived: re-arm for the next call
+                    sh->last_flag[et] = last;
                 }
                 epi_bar_sync();
-                if (sh->last_flag) {
+                for (int j = 0; j < nt; ++j) {
+                    if (!sh->last_flag[j]) continue;
                     __threadfence();
-                    for (int m = 0; m < m_valid; ++m) {
-                        float s = 0.0f;
-                        for (int cc = c_first; cc <= c_last; ++cc) {
-                            const int64_t b0 = sk_begin(U, G, cc);
-                            const int which = (b0 >= tile_first) ? 0 : 1;   // segment starts at its CTA's range start?
-                            const float* p = partials + ((size_t)2 * cc + which) * C::kSlotFloats;
-                            s += __ldcg(p + m * C::BN + r);
+                    const int tile = tc + j;
+                    const int64_t n = (int64_t)tile * C::BN + r;
+                    const float bv = (bias && n < N) ? __bfloat162float(bias[n]) : 0.0f;
+                    // 8 rows at a time: all loads of a batch are issued before the first add, so
+                    // the L2 round trips overlap instead of forming one long dependent chain
+                    const float* base = partials + (size_t)tile * C::kSlotFloats + r;
+                    const size_t band_stride = (size_t)plan.T * C::kSlotFloats;
+                    for (int m0 = 0; m0 < m_valid; m0 += 8) {
+                        float s[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) s[i] = 0.0f;
+                        for (int b = 0; b < plan.nbands; ++b) {         // bands in ascending K
+                            float t[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                t[i] = (m0 + i < m_valid) ? __ldcg(base + b * band_stride + (m0 + i) * C::BN) : 0.0f;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) s[i] += t[i];
                         }
-                        if (n < N) Y[(int64_t)m * N + n] = __float2bfloat16_rn(epilogue_rt<true>(s, bv, act));
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (m0 + i < m_valid && n < N)
+                                Y[(int64_t)(m0 + i) * N + n] = __float2bfloat16_rn(epilogue_rt<true>(s[i], bv, act));
                     }
                 }
+                epi_bar_sync();                           // last_flag is rewritten by the next chunk
             }
-            u += kb1 - kb0;
         }
         if (!ok && lane == 0) {
             atomicExch(status, kDevTimeout);

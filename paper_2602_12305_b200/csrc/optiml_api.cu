@@ -223,14 +223,11 @@ optiml_status_t launch_skinny_mp(optiml_handle_t h, const void* A, const void* B
     const CUtensorMap* ma = get_map(h, A, (uint64_t)M, (uint64_t)K, MP, 64);
     const CUtensorMap* mb = get_map(h, B, (uint64_t)K, (uint64_t)N, 64, 64);
     if (!ma || !mb) return OPTIML_ERR_CUDA;
-    const int64_t units = ceil_div64(N, C::BN) * ceil_div64(K, C::BK);
-    int G = h->num_sms;
-    if (units < G) G = (int)units;
-    // two scratch slots per CTA
-    if ((size_t)2 * G * C::kSlotFloats * sizeof(float) > kPartialBytes) return OPTIML_ERR_UNSUPPORTED;
-    gemm_skinny_umma_kernel<MP><<<G, C::kThreads, C::kSmemBytes, st>>>(*ma, *mb, (const __nv_bfloat16*)bias,
-                                                                       (__nv_bfloat16*)Y, M, N, K, act, h->partials,
-                                                                       h->counters, h->status);
+    const int64_t max_slots = kPartialBytes / (C::kSlotFloats * sizeof(float));
+    const SkinnyPlan plan = make_skinny_plan(ceil_div64(N, C::BN), ceil_div64(K, C::BK), h->num_sms, max_slots);
+    gemm_skinny_umma_kernel<MP><<<plan.G, C::kThreads, C::kSmemBytes, st>>>(
+        *ma, *mb, (const __nv_bfloat16*)bias, (__nv_bfloat16*)Y, M, N, K, act, plan, h->partials, h->counters,
+        h->status);
     h->launches += 1;
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
 }

@@ -1,0 +1,79 @@
+// Host-only self-test of the skinny kernel's schedule (SkinnyPlan / skinny_rect): for a
+// sweep of (column tiles, K blocks, CTAs) it checks that the rectangles cover every
+// (tile, K block) unit exactly once, that every tile is touched by exactly `nbands` CTAs
+// with distinct band indices (= distinct scratch slots), that no CTA is empty, and that
+// the largest rectangle stays close to the even share.  Built and run by the CPU
+// test-suite; needs no GPU.
+#include <cstdio>
+#include <set>
+#include <utility>
+#include <vector>
+
+#include "kernel_skinny.cuh"
+
+using namespace optiml;
+
+static double g_worst = 1.0;
+
+static int check(int64_t T, int64_t KB, int sms, int64_t max_slots) {
+    const SkinnyPlan p = make_skinny_plan(T, KB, sms, max_slots);
+    if (p.G != p.S * p.T + p.G1 + p.G2 || p.G < 1 || p.G > sms) return 1;
+    if (p.nbands != p.S + (p.G1 > 0) + (p.G2 > 0) || p.nbands < 1) return 2;
+    if (p.nbands > 1 && (int64_t)p.nbands * T > max_slots) return 3;
+    std::vector<int> cover((size_t)(T * KB), 0);
+    std::set<std::pair<int, int>> band_tile;
+    int64_t max_area = 0;
+    for (int c = 0; c < p.G; ++c) {
+        const SkinnyRect r = skinny_rect(p, c);
+        if (r.t0 < 0 || r.t1 > T || r.t0 >= r.t1 || r.kb0 < 0 || r.kb1 > KB || r.kb0 >= r.kb1) return 4;
+        if (r.band < 0 || r.band >= p.nbands) return 5;
+        for (int t = r.t0; t < r.t1; ++t) {
+            if (!band_tile.insert({r.band, t}).second) return 6;
+            for (int kb = r.kb0; kb < r.kb1; ++kb) cover[(size_t)t * KB + kb] += 1;
+        }
+        const int64_t area = (int64_t)(r.t1 - r.t0) * (r.kb1 - r.kb0);
+        if (area > max_area) max_area = area;
+    }
+    for (int v : cover)
+        if (v != 1) return 7;
+    if ((int64_t)band_tile.size() != (int64_t)p.nbands * T) return 8;
+    const int used = sms < T * KB ? sms : (int)(T * KB);
+    const double even = (double)(T * KB) / used;
+    const double ratio = (double)max_area / even;
+    const bool roomy = max_slots >= 3 * T;       // the scratch does not limit the banding
+    if (roomy && T * KB >= 8 * (int64_t)sms && ratio > g_worst) g_worst = ratio;
+    // with at least 8 units per CTA the banding must stay within 45 % of the even share (the
+    // worst cases are T just above the CTA count and very few K blocks; typical shapes are
+    // within a few per cent)
+    if (roomy && T * KB >= 8 * (int64_t)sms && ratio > 1.45) return 9;
+    return 0;
+}
+
+int main() {
+    const int64_t Ts[] = {1, 2, 3, 7, 37, 56, 64, 73, 74, 75, 111, 112, 147, 148, 149, 160, 200, 296, 300, 1000, 5000};
+    const int64_t KBs[] = {1, 2, 3, 5, 16, 17, 63, 64, 65, 128, 257};
+    const int smss[] = {1, 2, 7, 132, 148};
+    const int64_t slot_caps[] = {1024, 296};
+    int bad = 0, n = 0;
+    for (int64_t T : Ts)
+        for (int64_t KB : KBs)
+            for (int sms : smss)
+                for (int64_t cap : slot_caps) {
+                    const int rc = check(T, KB, sms, cap);
+                    ++n;
+                    if (rc) {
+                        std::printf("FAIL T=%lld KB=%lld sms=%d cap=%lld code=%d\n", (long long)T, (long long)KB, sms,
+                                    (long long)cap, rc);
+                        ++bad;
+                    }
+                }
+    const SkinnyPlan c3 = make_skinny_plan(112, 64, 148, 1024);
+    std::printf("c3 plan: S=%d k_split=%d G1=%d k_mid=%d G2=%d nbands=%d G=%d\n", c3.S, c3.k_split, c3.G1, c3.k_mid,
+                c3.G2, c3.nbands, c3.G);
+    const SkinnyPlan c2 = make_skinny_plan(64, 128, 148, 1024);
+    std::printf("c2 plan: S=%d k_split=%d G1=%d k_mid=%d G2=%d nbands=%d G=%d\n", c2.S, c2.k_split, c2.G1, c2.k_mid,
+                c2.G2, c2.nbands, c2.G);
+    std::printf("worst max-area / even-share ratio: %.3f\n", g_worst);
+    std::printf("%d plans checked, %d failed\n", n, bad);
+    return bad ? 1 : 0;
+}
