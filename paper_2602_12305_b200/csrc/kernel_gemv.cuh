@@ -11,6 +11,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "ptx_sm100.cuh"
 
 namespace optiml {
 
@@ -39,6 +40,10 @@ gemv_splitk_kernel(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __r
     for (int m = 0; m < MR; ++m)
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[m][j] = 0.0f;
+
+    // launched as a programmatic dependent: wait for the previous kernel before touching memory
+    ptx::griddep_wait();
+    ptx::griddep_launch_dependents();
 
     const __nv_bfloat16* bp = B + n;
     for (int kb = k_begin + warp; kb < k_end; kb += kGemvWarps * kGemvUnroll) {

@@ -100,6 +100,9 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     __syncthreads();
     ptx::tcgen05_fence_after_sync();
     const uint32_t tmem_base = sh->tmem_base;
+    // set-up above overlapped the previous kernel's tail; from here on global memory is touched
+    ptx::griddep_wait();
+    ptx::griddep_launch_dependents();
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer

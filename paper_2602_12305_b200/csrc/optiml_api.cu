@@ -11,6 +11,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <utility>
 
 #include "common.cuh"
 #include "kernel_f32.cuh"
@@ -142,6 +143,24 @@ int choose_variant(optiml_handle_t h, int64_t M, int64_t N, int64_t K, int dtype
 
 // ---------------------------------------------------------------- launches
 
+// Launch as a programmatic dependent of the previous kernel in the stream: this kernel's
+// CTAs may be scheduled, and run their set-up, while that kernel drains; the kernels call
+// griddepcontrol.wait before they touch global memory, so stream order is preserved.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 template <typename T>
 optiml_status_t launch_generic(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M,
                                int N, int K, int act, cudaStream_t st) {
@@ -191,9 +210,8 @@ optiml_status_t launch_f32(optiml_handle_t h, const void* A, const void* B, cons
 template <int MR>
 void launch_gemv_mr(const void* A, const void* B, const void* bias, void* Y, int M, int N, int K, int act, dim3 grid,
                     float* partials, unsigned int* counters, cudaStream_t st) {
-    gemv_splitk_kernel<MR><<<grid, kGemvThreads, 0, st>>>((const __nv_bfloat16*)A, (const __nv_bfloat16*)B,
-                                                          (const __nv_bfloat16*)bias, (__nv_bfloat16*)Y, M, N, K, act,
-                                                          partials, counters);
+    launch_pdl(gemv_splitk_kernel<MR>, grid, dim3(kGemvThreads), 0, st, (const __nv_bfloat16*)A,
+               (const __nv_bfloat16*)B, (const __nv_bfloat16*)bias, (__nv_bfloat16*)Y, M, N, K, act, partials, counters);
 }
 
 optiml_status_t launch_gemv(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
@@ -225,9 +243,8 @@ optiml_status_t launch_skinny_mp(optiml_handle_t h, const void* A, const void* B
     if (!ma || !mb) return OPTIML_ERR_CUDA;
     const int64_t max_slots = kPartialBytes / (C::kSlotFloats * sizeof(float));
     const SkinnyPlan plan = make_skinny_plan(ceil_div64(N, C::BN), ceil_div64(K, C::BK), h->num_sms, max_slots);
-    gemm_skinny_umma_kernel<MP><<<plan.G, C::kThreads, C::kSmemBytes, st>>>(
-        *ma, *mb, (const __nv_bfloat16*)bias, (__nv_bfloat16*)Y, M, N, K, act, plan, h->partials, h->counters,
-        h->status);
+    launch_pdl(gemm_skinny_umma_kernel<MP>, dim3(plan.G), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb,
+               (const __nv_bfloat16*)bias, (__nv_bfloat16*)Y, M, N, K, act, plan, h->partials, h->counters, h->status);
     h->launches += 1;
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
 }
@@ -252,13 +269,16 @@ optiml_status_t launch_umma(optiml_handle_t h, const void* A, const void* B, con
     __nv_bfloat16* y = (__nv_bfloat16*)Y;
     switch (act) {
     case OPTIML_ACT_RELU:
-        gemm_umma_kernel<kActRelu><<<grid, C::kThreads, C::kSmemBytes, st>>>(*ma, *mb, bi, y, M, N, K, h->status);
+        launch_pdl(gemm_umma_kernel<kActRelu>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, bi, y, M, N, K,
+                   h->status);
         break;
     case OPTIML_ACT_GELU_TANH:
-        gemm_umma_kernel<kActGeluTanh><<<grid, C::kThreads, C::kSmemBytes, st>>>(*ma, *mb, bi, y, M, N, K, h->status);
+        launch_pdl(gemm_umma_kernel<kActGeluTanh>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, bi, y, M, N, K,
+                   h->status);
         break;
     default:
-        gemm_umma_kernel<kActNone><<<grid, C::kThreads, C::kSmemBytes, st>>>(*ma, *mb, bi, y, M, N, K, h->status);
+        launch_pdl(gemm_umma_kernel<kActNone>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, bi, y, M, N, K,
+                   h->status);
         break;
     }
     h->launches += 1;

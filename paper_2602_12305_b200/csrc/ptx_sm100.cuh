@@ -66,6 +66,18 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     }
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+
+// Kernels launched with the programmatic-stream-serialization attribute may start while the
+// previous kernel in the stream is still draining.  griddep_wait() blocks until every
+// earlier kernel has completed and its writes are visible: nothing that reads or writes
+// global memory may come before it.  griddep_launch_dependents() lets the next kernel's
+// CTAs be scheduled as soon as SM resources free up.  Both are no-ops for a plain launch.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---------------------------------------------------------------- proxies / fences
 
 // Make generic-proxy writes to shared memory visible to the async proxy (TMA, tcgen05).
