@@ -127,15 +127,17 @@ bool variant_supports(int v, int64_t M, int64_t N, int64_t K, int dtype, bool al
     }
 }
 
-// Shape-based choice.  fp32 goes to the FMA tiles.  bf16: M <= 4 is a pure stream over B
-// (CUDA-core split-K), M <= 64 is still bandwidth-bound but needs tensor-core MACs
+// Shape-based choice.  fp32 goes to the FMA tiles.  bf16: M = 1 is a pure stream over B
+// (CUDA-core split-K; measured 5.5 TB/s against 4.9 TB/s for the tensor-core stream; at
+// M = 4 the FMA pipes already fall behind: 81 us against 28 us on 4 x 8192 x 8192),
+// M <= 64 is still bandwidth-bound but needs tensor-core MACs
 // (stream-K tcgen05 with N as the MMA M dimension), larger M is compute-bound.
 int choose_variant(optiml_handle_t h, int64_t M, int64_t N, int64_t K, int dtype, bool al16) {
     if (h->forced != OPTIML_VARIANT_AUTO) return h->forced;
     if (dtype == OPTIML_F32)
         return variant_supports(OPTIML_VARIANT_F32_TILED, M, N, K, dtype, al16) ? OPTIML_VARIANT_F32_TILED
                                                                                  : OPTIML_VARIANT_GENERIC;
-    if (M <= 4 && variant_supports(OPTIML_VARIANT_GEMV_SPLITK, M, N, K, dtype, al16)) return OPTIML_VARIANT_GEMV_SPLITK;
+    if (M == 1 && variant_supports(OPTIML_VARIANT_GEMV_SPLITK, M, N, K, dtype, al16)) return OPTIML_VARIANT_GEMV_SPLITK;
     if (M <= 64 && variant_supports(OPTIML_VARIANT_SKINNY_UMMA, M, N, K, dtype, al16)) return OPTIML_VARIANT_SKINNY_UMMA;
     if (variant_supports(OPTIML_VARIANT_UMMA, M, N, K, dtype, al16)) return OPTIML_VARIANT_UMMA;
     return OPTIML_VARIANT_GENERIC;
@@ -218,9 +220,9 @@ optiml_status_t launch_gemv(optiml_handle_t h, const void* A, const void* B, con
                             int K, int act, cudaStream_t st) {
     const int MR = M == 1 ? 1 : (M == 2 ? 2 : 4);
     const int64_t col_blocks = ceil_div64(N, kGemvCols);
-    // K slices: fill every SM with two CTAs in one wave, keep at least 64 rows per slice,
+    // K slices: fill every SM with its resident CTAs in one wave, keep at least 64 rows per slice,
     // stay inside the scratch and the 65535 limit of gridDim.y.
-    int64_t S = (2 * (int64_t)h->num_sms) / col_blocks;
+    int64_t S = (gemv_ctas_per_sm(MR) * (int64_t)h->num_sms) / col_blocks;
     if (S > K / 64) S = K / 64;
     const int64_t per_slice = (int64_t)MR * kGemvCols * sizeof(float);
     if (S * col_blocks * per_slice > (int64_t)kPartialBytes) S = kPartialBytes / (col_blocks * per_slice);
