@@ -264,23 +264,24 @@ optiml_status_t launch_umma(optiml_handle_t h, const void* A, const void* B, con
     using C = UmmaCfg;
     const CUtensorMap* ma = get_map(h, A, (uint64_t)M, (uint64_t)K, C::BM, 64);
     const CUtensorMap* mb = get_map(h, B, (uint64_t)K, (uint64_t)N, 64, 64);
-    if (!ma || !mb) return OPTIML_ERR_CUDA;
-    const int64_t tiles = ceil_div64(M, C::BM) * ceil_div64(N, C::BN);
-    const int grid = (int)(tiles < h->num_sms ? tiles : h->num_sms);
+    const CUtensorMap* my = get_map(h, Y, (uint64_t)M, (uint64_t)N, 32, 64);
+    if (!ma || !mb || !my) return OPTIML_ERR_CUDA;
+    const UmmaPlan plan = make_umma_plan(M, N, K, h->num_sms);
+    if ((size_t)plan.rem_tiles * plan.split * C::BM * C::BN * sizeof(float) > kPartialBytes) return OPTIML_ERR_UNSUPPORTED;
+    const int grid = plan.grid;
     const __nv_bfloat16* bi = (const __nv_bfloat16*)bias;
-    __nv_bfloat16* y = (__nv_bfloat16*)Y;
     switch (act) {
     case OPTIML_ACT_RELU:
-        launch_pdl(gemm_umma_kernel<kActRelu>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, bi, y, M, N, K,
-                   h->status);
+        launch_pdl(gemm_umma_kernel<kActRelu>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
+                   plan, h->partials, h->counters, h->status);
         break;
     case OPTIML_ACT_GELU_TANH:
-        launch_pdl(gemm_umma_kernel<kActGeluTanh>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, bi, y, M, N, K,
-                   h->status);
+        launch_pdl(gemm_umma_kernel<kActGeluTanh>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
+                   plan, h->partials, h->counters, h->status);
         break;
     default:
-        launch_pdl(gemm_umma_kernel<kActNone>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, bi, y, M, N, K,
-                   h->status);
+        launch_pdl(gemm_umma_kernel<kActNone>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
+                   plan, h->partials, h->counters, h->status);
         break;
     }
     h->launches += 1;

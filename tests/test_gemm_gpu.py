@@ -73,7 +73,9 @@ def test_skinny_variant(handle, M, N, K, act):
 
 
 @pytest.mark.parametrize("M,N,K", [(128, 256, 64), (128, 256, 512), (300, 520, 200), (130, 264, 72), (1, 8, 8),
-                                   (1024, 1024, 512),
+                                   (1024, 1024, 512),     # 32 tiles: each cut into 2 K slices
+                                   (256, 520, 4096),      # 6 tiles, 8 K slices each
+                                   (2432, 4096, 256),     # 304 tiles = 2 rounds + 8 tiles cut into 4 K slices
                                    (2048, 4096, 128)])   # 256 tiles: more than one tile per CTA
 @pytest.mark.parametrize("act", [RELU, GELU])
 def test_umma_variant(handle, M, N, K, act):
