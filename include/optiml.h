@@ -60,7 +60,8 @@ typedef enum {
     OPTIML_VARIANT_GEMV_SPLITK = 2, /* bf16, M <= 4: split-K streaming with 128-bit loads, N % 8 == 0    */
     OPTIML_VARIANT_SKINNY_UMMA = 3, /* bf16, M <= 128: stream-K over B with tcgen05 (N is the MMA M dim) */
     OPTIML_VARIANT_UMMA = 4,        /* bf16: persistent TMA + tcgen05 + TMEM tiles, N % 8 == K % 8 == 0  */
-    OPTIML_VARIANT_COUNT = 5
+    OPTIML_VARIANT_UMMA_2CTA = 5,   /* bf16: the same with CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles) */
+    OPTIML_VARIANT_COUNT = 6
 } optiml_variant_t;
 
 /*

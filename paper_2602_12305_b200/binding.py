@@ -15,7 +15,8 @@ import torch
 F32, BF16 = 0, 1
 ACT_NONE, ACT_RELU, ACT_GELU_TANH = 0, 1, 2
 VARIANT_AUTO, VARIANT_GENERIC, VARIANT_F32_TILED, VARIANT_GEMV_SPLITK, VARIANT_SKINNY_UMMA, VARIANT_UMMA = -1, 0, 1, 2, 3, 4
-VARIANT_COUNT = 5
+VARIANT_UMMA_2CTA = 5
+VARIANT_COUNT = 6
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ARCH, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(8)
 

@@ -19,6 +19,7 @@
 #include "kernel_generic.cuh"
 #include "kernel_skinny.cuh"
 #include "kernel_umma.cuh"
+#include "kernel_umma2.cuh"
 
 using namespace optiml;
 
@@ -120,6 +121,7 @@ bool variant_supports(int v, int64_t M, int64_t N, int64_t K, int dtype, bool al
         return dtype == OPTIML_BF16 && M <= 128 && N % 8 == 0 && K % 8 == 0 && al16 &&
                ceil_div64(N, 128) <= kNumCounters;
     case OPTIML_VARIANT_UMMA:
+    case OPTIML_VARIANT_UMMA_2CTA:
         return dtype == OPTIML_BF16 && N % 8 == 0 && K % 8 == 0 && al16 &&
                ceil_div64(M, UmmaCfg::BM) * ceil_div64(N, UmmaCfg::BN) < (int64_t)1 << 31;
     default:
@@ -139,6 +141,8 @@ int choose_variant(optiml_handle_t h, int64_t M, int64_t N, int64_t K, int dtype
                                                                                  : OPTIML_VARIANT_GENERIC;
     if (M == 1 && variant_supports(OPTIML_VARIANT_GEMV_SPLITK, M, N, K, dtype, al16)) return OPTIML_VARIANT_GEMV_SPLITK;
     if (M <= 64 && variant_supports(OPTIML_VARIANT_SKINNY_UMMA, M, N, K, dtype, al16)) return OPTIML_VARIANT_SKINNY_UMMA;
+    // above 128 rows a CTA pair shares one 256 x 256 tile (a third less operand traffic per flop)
+    if (M > 128 && variant_supports(OPTIML_VARIANT_UMMA_2CTA, M, N, K, dtype, al16)) return OPTIML_VARIANT_UMMA_2CTA;
     if (variant_supports(OPTIML_VARIANT_UMMA, M, N, K, dtype, al16)) return OPTIML_VARIANT_UMMA;
     return OPTIML_VARIANT_GENERIC;
 }
@@ -288,6 +292,36 @@ optiml_status_t launch_umma(optiml_handle_t h, const void* A, const void* B, con
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
 }
 
+optiml_status_t launch_umma2(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
+                             int K, int act, cudaStream_t st) {
+    using C = Umma2Cfg;
+    const CUtensorMap* ma = get_map(h, A, (uint64_t)M, (uint64_t)K, 128, 64);
+    const CUtensorMap* mb = get_map(h, B, (uint64_t)K, (uint64_t)N, 64, 64);
+    const CUtensorMap* my = get_map(h, Y, (uint64_t)M, (uint64_t)N, 32, 64);
+    if (!ma || !mb || !my) return OPTIML_ERR_CUDA;
+    const UmmaPlan plan = make_umma2_plan(M, N, K, h->num_sms);
+    if ((size_t)plan.rem_tiles * plan.split * C::BM * C::BN * sizeof(float) > kPartialBytes) return OPTIML_ERR_UNSUPPORTED;
+    if (2 * plan.rem_tiles > kNumCounters) return OPTIML_ERR_UNSUPPORTED;
+    const dim3 grid(2 * plan.grid);          // CTA pairs: the kernel is compiled with cluster dimensions (2, 1, 1)
+    const __nv_bfloat16* bi = (const __nv_bfloat16*)bias;
+    switch (act) {
+    case OPTIML_ACT_RELU:
+        launch_pdl(gemm_umma2_kernel<kActRelu>, grid, dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
+                   plan, h->partials, h->counters, h->status);
+        break;
+    case OPTIML_ACT_GELU_TANH:
+        launch_pdl(gemm_umma2_kernel<kActGeluTanh>, grid, dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N,
+                   K, plan, h->partials, h->counters, h->status);
+        break;
+    default:
+        launch_pdl(gemm_umma2_kernel<kActNone>, grid, dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
+                   plan, h->partials, h->counters, h->status);
+        break;
+    }
+    h->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
 template <typename F>
 bool set_smem(F* fn, int bytes) {
     return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
@@ -298,6 +332,9 @@ bool configure_kernels() {
     ok &= set_smem(gemm_umma_kernel<kActNone>, UmmaCfg::kSmemBytes);
     ok &= set_smem(gemm_umma_kernel<kActRelu>, UmmaCfg::kSmemBytes);
     ok &= set_smem(gemm_umma_kernel<kActGeluTanh>, UmmaCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2_kernel<kActNone>, Umma2Cfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2_kernel<kActRelu>, Umma2Cfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2_kernel<kActGeluTanh>, Umma2Cfg::kSmemBytes);
     ok &= set_smem(gemm_skinny_umma_kernel<16>, SkinnyCfg<16>::kSmemBytes);
     ok &= set_smem(gemm_skinny_umma_kernel<32>, SkinnyCfg<32>::kSmemBytes);
     ok &= set_smem(gemm_skinny_umma_kernel<64>, SkinnyCfg<64>::kSmemBytes);
@@ -409,6 +446,8 @@ optiml_status_t optiml_gemm_epilogue(optiml_handle_t h, const void* A, const voi
         return launch_skinny(h, A, B, bias, Y, m, n, k, (int)act, st);
     case OPTIML_VARIANT_UMMA:
         return launch_umma(h, A, B, bias, Y, m, n, k, (int)act, st);
+    case OPTIML_VARIANT_UMMA_2CTA:
+        return launch_umma2(h, A, B, bias, Y, m, n, k, (int)act, st);
     default:
         return dtype == OPTIML_F32 ? launch_generic<float>(h, A, B, bias, Y, m, n, k, (int)act, st)
                                    : launch_generic<__nv_bfloat16>(h, A, B, bias, Y, m, n, k, (int)act, st);
@@ -499,6 +538,7 @@ const char* optiml_variant_name(int variant) {
     case OPTIML_VARIANT_GEMV_SPLITK: return "gemv_splitk_stream";
     case OPTIML_VARIANT_SKINNY_UMMA: return "skinny_streamk_tcgen05";
     case OPTIML_VARIANT_UMMA: return "persistent_tcgen05";
+    case OPTIML_VARIANT_UMMA_2CTA: return "persistent_tcgen05_cta_pair";
     default: return "unknown";
     }
 }

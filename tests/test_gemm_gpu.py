@@ -78,13 +78,15 @@ def test_skinny_variant(handle, M, N, K, act):
                                    (2432, 4096, 256),     # 304 tiles = 2 rounds + 8 tiles cut into 4 K slices
                                    (2048, 4096, 128)])   # 256 tiles: more than one tile per CTA
 @pytest.mark.parametrize("act", [RELU, GELU])
-def test_umma_variant(handle, M, N, K, act):
-    parity(handle, synth.make_case("c4", M=M, N=N, K=K, act=act), V.VARIANT_UMMA)
+@pytest.mark.parametrize("variant", [V.VARIANT_UMMA, V.VARIANT_UMMA_2CTA])
+def test_umma_variant(handle, M, N, K, act, variant):
+    parity(handle, synth.make_case("c4", M=M, N=N, K=K, act=act), variant)
 
 
 def test_null_bias_and_act_none(handle):
     for variant, name, shape in ((V.VARIANT_F32_TILED, "c1", (64, 64, 64)), (V.VARIANT_GEMV_SPLITK, "c2", (1, 512, 512)),
                                  (V.VARIANT_SKINNY_UMMA, "c3", (16, 512, 512)), (V.VARIANT_UMMA, "c4", (256, 512, 256)),
+                                 (V.VARIANT_UMMA_2CTA, "c4", (256, 512, 256)),
                                  (V.VARIANT_GENERIC, "c4", (50, 60, 70))):
         c = synth.make_case(name, M=shape[0], N=shape[1], K=shape[2], act=NONE)
         c.bias = None
@@ -97,7 +99,8 @@ def test_null_bias_and_act_none(handle):
     (V.VARIANT_GENERIC, F32, 70, 90, 300), (V.VARIANT_GENERIC, BF16, 70, 90, 300),
     (V.VARIANT_F32_TILED, F32, 96, 160, 512), (V.VARIANT_GEMV_SPLITK, BF16, 1, 1024, 4096),
     (V.VARIANT_GEMV_SPLITK, BF16, 4, 520, 1000), (V.VARIANT_SKINNY_UMMA, BF16, 16, 1160, 1096),
-    (V.VARIANT_SKINNY_UMMA, BF16, 48, 648, 2048), (V.VARIANT_UMMA, BF16, 384, 776, 1024)])
+    (V.VARIANT_SKINNY_UMMA, BF16, 48, 648, 2048), (V.VARIANT_UMMA, BF16, 384, 776, 1024),
+    (V.VARIANT_UMMA_2CTA, BF16, 384, 776, 1024), (V.VARIANT_UMMA_2CTA, BF16, 1000, 520, 320)])
 @pytest.mark.parametrize("act", [NONE, RELU])
 def test_integer_inputs_are_bit_exact(handle, variant, dtype, M, N, K, act):
     c = synth.integer_case(M, N, K, dtype, act, seed=11)
@@ -116,7 +119,7 @@ def test_permutation_B_on_the_tensor_core_path(handle):
     Bm[perm, np.arange(K)] = 1.0
     c.B = synth.round_to_bf16_bits(Bm).reshape(-1)
     c.bias = None
-    for variant in (V.VARIANT_UMMA, V.VARIANT_SKINNY_UMMA, V.VARIANT_GENERIC):
+    for variant in (V.VARIANT_UMMA, V.VARIANT_UMMA_2CTA, V.VARIANT_SKINNY_UMMA, V.VARIANT_GENERIC):
         if variant == V.VARIANT_SKINNY_UMMA:
             c2 = synth.Case("perm", 64, K, K, BF16, NONE, c.A[:64 * K], c.B, None)
         else:
@@ -164,7 +167,7 @@ def test_c3_full(handle):
 @pytest.mark.parametrize("name", ["c4", "c5"])
 def test_c4_c5_sampled(handle, name):
     c = synth.make_case(name)
-    assert handle.select_variant(c.M, c.N, c.K, c.dtype) == V.VARIANT_UMMA
+    assert handle.select_variant(c.M, c.N, c.K, c.dtype) == V.VARIANT_UMMA_2CTA
     bits, y = H.run_case(handle, c)
     rows = sample_indices(c.M, 128, 160, 1)
     cols = sample_indices(c.N, 256, 288, 2)
@@ -193,8 +196,9 @@ def test_dispatcher_choices(handle):
     assert sel(255, 255, 255, F32) == V.VARIANT_GENERIC
     assert sel(1, 8192, 8192, BF16) in (V.VARIANT_GEMV_SPLITK, V.VARIANT_SKINNY_UMMA)
     assert sel(16, 14336, 4096, BF16) == V.VARIANT_SKINNY_UMMA
-    assert sel(4096, 4096, 4096, BF16) == V.VARIANT_UMMA
-    assert sel(8192, 8192, 16384, BF16) == V.VARIANT_UMMA
+    assert sel(4096, 4096, 4096, BF16) == V.VARIANT_UMMA_2CTA
+    assert sel(8192, 8192, 16384, BF16) == V.VARIANT_UMMA_2CTA
+    assert sel(128, 4096, 4096, BF16) == V.VARIANT_UMMA
     assert sel(4096, 4100, 4096, BF16) == V.VARIANT_GENERIC      # N % 8 != 0
     assert sel(0, 1, 1, BF16) == -1
 
@@ -245,7 +249,8 @@ def test_error_codes(handle):
 @pytest.mark.parametrize("variant,name,M,N,K", [(V.VARIANT_F32_TILED, "c1", 96, 128, 256),
                                                 (V.VARIANT_GEMV_SPLITK, "c2", 2, 1024, 2048),
                                                 (V.VARIANT_SKINNY_UMMA, "c3", 16, 1160, 1096),
-                                                (V.VARIANT_UMMA, "c4", 384, 512, 512)])
+                                                (V.VARIANT_UMMA, "c4", 384, 512, 512),
+                                                (V.VARIANT_UMMA_2CTA, "c4", 384, 512, 512)])
 def test_metamorphic_relations(handle, variant, name, M, N, K):
     c = synth.make_case(name, M=M, N=N, K=K, act=RELU)
     handle.force_variant(variant)
