@@ -35,6 +35,8 @@
 // All mbarrier waits are bounded; see kernel_umma.cuh for the tear-down protocol.
 #pragma once
 
+#include <math.h>
+
 #include "common.cuh"
 #include "ptx_sm100.cuh"
 
@@ -129,10 +131,17 @@ __host__ __device__ __forceinline__ SkinnyRect skinny_rect(const SkinnyPlan& p, 
     return r;
 }
 
-// Best balanced banding for `num_sms` CTAs.  cost = the largest rectangle area (K blocks
-// x column tiles) any CTA has to stream; ties go to fewer bands (fewer partial tiles).
-// `max_slots` bounds bands * T, the partial tiles the scratch can hold.
-inline SkinnyPlan make_skinny_plan(int64_t tiles, int64_t kblocks, int num_sms, int64_t max_slots) {
+// Best banding for `num_sms` CTAs; `max_slots` bounds bands * T, the partial tiles the
+// scratch can hold.  With unit_us <= 0 the cost of a plan is the largest rectangle area
+// (K blocks x column tiles) any CTA has to stream, ties going to fewer bands.  With
+// unit_us > 0 (the time one CTA needs to stream one unit at the per-SM rate) the cost is an
+// estimated run time, fitted to measurements on B200: a CTA streams at most about 58 GB/s,
+// all of them together at most about 6.5 TB/s (= 112 CTAs' worth), the two limits combine
+// like a 4-norm, and any split along K costs about 2.5 us for the partial-tile round trip.
+// So 112 whole tiles on 112 SMs beat a perfectly balanced two-band plan for a 118 MB
+// problem, while a 470 MB problem is better off balanced.
+inline SkinnyPlan make_skinny_plan(int64_t tiles, int64_t kblocks, int num_sms, int64_t max_slots,
+                                   double unit_us = 0.0) {
     const int64_t T = tiles, KB = kblocks;
     SkinnyPlan best;
     best.T = (int)T;
@@ -145,7 +154,14 @@ inline SkinnyPlan make_skinny_plan(int64_t tiles, int64_t kblocks, int num_sms, 
     best.G2 = 0;
     best.nbands = 1;
     best.G = best.G1;
-    int64_t best_cost = ((T + best.G1 - 1) / best.G1) * KB;
+    auto estimate = [&](int64_t area, int nb) -> double {
+        if (unit_us <= 0.0) return (double)area;
+        const double t_sm = (double)area * unit_us;
+        const double t_dram = (double)(T * KB) * unit_us / 112.0;
+        const double t = sqrt(sqrt(t_sm * t_sm * t_sm * t_sm + t_dram * t_dram * t_dram * t_dram));
+        return t + (nb > 1 ? 2.5 : 0.0);
+    };
+    double best_cost = estimate(((T + best.G1 - 1) / best.G1) * KB, 1);
 
     auto consider = [&](int S, int64_t k_split, int G1, int64_t k_mid, int G2) {
         const int nb = S + (G1 > 0) + (G2 > 0);
@@ -155,15 +171,16 @@ inline SkinnyPlan make_skinny_plan(int64_t tiles, int64_t kblocks, int num_sms, 
         if (G2 > 0 && KB <= k_mid) return;
         if (G2 == 0 && k_mid != KB) return;
         if (G1 == 0 && (k_split != KB || G2 != 0)) return;
-        int64_t cost = S > 0 ? (k_split + S - 1) / S : 0;
+        int64_t area = S > 0 ? (k_split + S - 1) / S : 0;
         if (G1 > 0) {
             const int64_t c1 = ((T + G1 - 1) / G1) * (k_mid - k_split);
-            if (c1 > cost) cost = c1;
+            if (c1 > area) area = c1;
         }
         if (G2 > 0) {
             const int64_t c2 = ((T + G2 - 1) / G2) * (KB - k_mid);
-            if (c2 > cost) cost = c2;
+            if (c2 > area) area = c2;
         }
+        const double cost = estimate(area, nb);
         if (cost < best_cost || (cost == best_cost && nb < best.nbands)) {
             best_cost = cost;
             best.S = S;

@@ -248,7 +248,9 @@ optiml_status_t launch_skinny_mp(optiml_handle_t h, const void* A, const void* B
     const CUtensorMap* mb = get_map(h, B, (uint64_t)K, (uint64_t)N, 64, 64);
     if (!ma || !mb) return OPTIML_ERR_CUDA;
     const int64_t max_slots = kPartialBytes / (C::kSlotFloats * sizeof(float));
-    const SkinnyPlan plan = make_skinny_plan(ceil_div64(N, C::BN), ceil_div64(K, C::BK), h->num_sms, max_slots);
+    // one unit = one K block of one column tile; a CTA streams it at about 58 GB/s
+    const double unit_us = (double)(C::kBBytes + C::kABytes) / 58.0e3;
+    const SkinnyPlan plan = make_skinny_plan(ceil_div64(N, C::BN), ceil_div64(K, C::BK), h->num_sms, max_slots, unit_us);
     launch_pdl(gemm_skinny_umma_kernel<MP>, dim3(plan.G), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb,
                (const __nv_bfloat16*)bias, (__nv_bfloat16*)Y, M, N, K, act, plan, h->partials, h->counters, h->status);
     h->launches += 1;

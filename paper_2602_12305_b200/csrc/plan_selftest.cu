@@ -67,6 +67,12 @@ int main() {
                         ++bad;
                     }
                 }
+    // with the run-time model (192-row units of 51 KiB: 0.9 us each) the 16 x 14336 x 4096
+    // problem runs as 112 whole tiles, four times the K as two balanced bands
+    const SkinnyPlan c3t = make_skinny_plan(112, 22, 148, 1024, 0.9);
+    const SkinnyPlan c3l = make_skinny_plan(112, 86, 148, 1024, 0.9);
+    std::printf("c3 timed plan: nbands=%d G=%d; 4x K: nbands=%d G=%d\n", c3t.nbands, c3t.G, c3l.nbands, c3l.G);
+    if (c3t.nbands != 1 || c3t.G != 112 || c3l.nbands != 2 || c3l.G != 148) ++bad;
     const SkinnyPlan c3 = make_skinny_plan(112, 64, 148, 1024);
     std::printf("c3 plan: S=%d k_split=%d G1=%d k_mid=%d G2=%d nbands=%d G=%d\n", c3.S, c3.k_split, c3.G1, c3.k_mid,
                 c3.G2, c3.nbands, c3.G);
