@@ -47,7 +47,7 @@ FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel,
 # from the ncu captures summarised under profiles/; None = not captured for the current kernel.
-NCU_TRAFFIC_BYTES = {"c1": 542464, "c2": 137815296, "c3": None, "c4": None, "c5": None}
+NCU_TRAFFIC_BYTES = {"c1": 542208, "c2": 137838336, "c3": 121811968, "c4": 110100992, "c5": 2564892440}
 
 
 def load_peaks():
