@@ -72,6 +72,14 @@ __device__ __forceinline__ uint4 ld_stream_v4(const void* p) {
     return v;
 }
 
+// Record a bounded wait that gave up: low byte = status, next byte = which wait (1 producer
+// waiting for a free stage, 2 MMA waiting for a free accumulator, 3 MMA waiting for the A
+// tile, 4 MMA waiting for a filled stage, 5 epilogue waiting for an accumulator), upper
+// half = CTA index.  The first report wins.
+__device__ __forceinline__ void report_timeout(int* status, int site) {
+    atomicCAS(status, kDevOk, kDevTimeout | (site << 8) | ((int)(blockIdx.x & 0x7FFF) << 16));
+}
+
 __host__ __device__ __forceinline__ int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
 }  // namespace optiml

@@ -275,6 +275,7 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             const uint64_t pol_keep = ptx::policy_evict_last();      // A is re-read by every CTA
             uint32_t it = 0, ait = 0;
             bool ok = true;
+            int site = 0;
             for (int tc = rect.t0; tc < rect.t1 && ok; tc += C::kAcc) {
                 const int nt = min(C::kAcc, rect.t1 - tc);
                 for (int kb = rect.kb0; kb < rect.kb1 && ok; ++kb, ++ait) {
@@ -286,7 +287,7 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                                               kb * C::BK + u * 64, 0, pol_keep);
                     for (int j = 0; j < nt; ++j, ++it) {
                         const int s = it % C::kStages;
-                        if (sh->abort || !ptx::mbar_wait(&sh->empty[s], ((it / C::kStages) & 1) ^ 1)) { ok = false; break; }
+                        if (sh->abort || (site = 1, !ptx::mbar_wait(&sh->empty[s], ((it / C::kStages) & 1) ^ 1))) { ok = false; break; }
                         uint8_t* b_dst = ring + s * C::kBBytes;
                         ptx::mbar_arrive_expect_tx(&sh->full[s], C::kBBytes);
 #pragma unroll
@@ -300,7 +301,7 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 }
             }
             if (!ok) {
-                atomicExch(status, kDevTimeout);
+                report_timeout(status, site);
                 sh->abort = 1;
                 // copies already issued must land before the CTA may exit
                 const uint32_t n_back = it < (uint32_t)C::kStages ? it : (uint32_t)C::kStages;
@@ -321,18 +322,19 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             constexpr uint32_t idesc = ptx::umma_idesc_bf16(C::BN, MP, /*a_mn_major=*/true, /*b_mn_major=*/false);
             uint32_t it = 0, ait = 0, chunk_it = 0;
             bool ok = true;
+            int site = 0;
             for (int tc = rect.t0; tc < rect.t1 && ok; tc += C::kAcc, ++chunk_it) {
                 const int nt = min(C::kAcc, rect.t1 - tc);
                 const int half = chunk_it & 1;
-                if (sh->abort || !ptx::mbar_wait(&sh->tmem_empty[half], ((chunk_it >> 1) & 1) ^ 1)) { ok = false; break; }
+                if (sh->abort || (site = 2, !ptx::mbar_wait(&sh->tmem_empty[half], ((chunk_it >> 1) & 1) ^ 1))) { ok = false; break; }
                 ptx::tcgen05_fence_after_sync();
                 for (int kb = rect.kb0; kb < rect.kb1 && ok; ++kb, ++ait) {
                     const int sa = ait % C::kAStages;
-                    if (sh->abort || !ptx::mbar_wait(&sh->a_full[sa], (ait / C::kAStages) & 1)) { ok = false; break; }
+                    if (sh->abort || (site = 3, !ptx::mbar_wait(&sh->a_full[sa], (ait / C::kAStages) & 1))) { ok = false; break; }
                     const uint32_t a_addr = aring_base + sa * C::kABytes;            // tile of A
                     for (int j = 0; j < nt; ++j, ++it) {
                         const int s = it % C::kStages;
-                        if (sh->abort || !ptx::mbar_wait(&sh->full[s], (it / C::kStages) & 1)) { ok = false; break; }
+                        if (sh->abort || (site = 4, !ptx::mbar_wait(&sh->full[s], (it / C::kStages) & 1))) { ok = false; break; }
                         ptx::tcgen05_fence_after_sync();
                         const uint32_t b_addr = ring_base + s * C::kBBytes;          // tile of B
                         const uint32_t d_tmem = tmem_base + (half * C::kAcc + j) * MP;
@@ -350,7 +352,7 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 if (ok) ptx::umma_commit(&sh->tmem_full[half]);
             }
             if (!ok) {
-                atomicExch(status, kDevTimeout);
+                report_timeout(status, site);
                 sh->abort = 1;
             }
             ptx::umma_commit(&sh->drain);
@@ -453,7 +455,7 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             }
         }
         if (!ok && lane == 0) {
-            atomicExch(status, kDevTimeout);
+            report_timeout(status, 5);
             sh->abort = 1;
         }
     }

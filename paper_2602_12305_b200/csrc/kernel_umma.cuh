@@ -185,13 +185,14 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             ptx::prefetch_tensormap(&map_b);
             uint32_t it = 0;
             bool ok = true;
+            int site = 0;
             UmmaWork w;
             for (int wi = 0; ok && umma_work_item(plan, blockIdx.x, wi, w); ++wi) {
                 const int tm = w.tm, tn = w.tn;
                 for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
                     const int s = it % C::kStages;
                     const uint32_t ph = (it / C::kStages) & 1;
-                    if (sh->abort || !ptx::mbar_wait(&sh->empty[s], ph ^ 1)) { ok = false; break; }
+                    if (sh->abort || (site = 1, !ptx::mbar_wait(&sh->empty[s], ph ^ 1))) { ok = false; break; }
                     uint8_t* a_dst = ring + s * C::kStageBytes;
                     uint8_t* b_dst = a_dst + C::kABytes;
                     ptx::mbar_arrive_expect_tx(&sh->full[s], C::kStageBytes);
@@ -203,7 +204,7 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 }
             }
             if (!ok) {
-                atomicExch(status, kDevTimeout);
+                report_timeout(status, site);
                 sh->abort = 1;
                 // copies already issued must land before the CTA may exit
                 const uint32_t n_back = it < (uint32_t)C::kStages ? it : (uint32_t)C::kStages;
@@ -219,17 +220,18 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             constexpr uint32_t idesc = ptx::umma_idesc_bf16(C::BM, C::BN, /*a_mn_major=*/false, /*b_mn_major=*/true);
             uint32_t it = 0, tile_it = 0;
             bool ok = true;
+            int site = 0;
             UmmaWork w;
             for (int wi = 0; ok && umma_work_item(plan, blockIdx.x, wi, w); ++wi, ++tile_it) {
                 const int a = tile_it & 1;
                 const uint32_t aph = (tile_it >> 1) & 1;
-                if (sh->abort || !ptx::mbar_wait(&sh->tmem_empty[a], aph ^ 1)) { ok = false; break; }
+                if (sh->abort || (site = 2, !ptx::mbar_wait(&sh->tmem_empty[a], aph ^ 1))) { ok = false; break; }
                 ptx::tcgen05_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + a * C::BN;
                 for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
                     const int s = it % C::kStages;
                     const uint32_t ph = (it / C::kStages) & 1;
-                    if (sh->abort || !ptx::mbar_wait(&sh->full[s], ph)) { ok = false; break; }
+                    if (sh->abort || (site = 4, !ptx::mbar_wait(&sh->full[s], ph))) { ok = false; break; }
                     ptx::tcgen05_fence_after_sync();
                     const uint32_t a_addr = ring_base + s * C::kStageBytes;
                     const uint32_t b_addr = a_addr + C::kABytes;
@@ -246,7 +248,7 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 if (ok) ptx::umma_commit(&sh->tmem_full[a]);
             }
             if (!ok) {
-                atomicExch(status, kDevTimeout);
+                report_timeout(status, site);
                 sh->abort = 1;
             }
             // nothing may be in flight on the tensor pipe when TMEM is freed
@@ -408,7 +410,7 @@ gemm_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         if (lane == 0) ptx::tma_store_wait_all<0>();
         __syncwarp();
         if (!ok && lane == 0) {
-            atomicExch(status, kDevTimeout);
+            report_timeout(status, 5);
             sh->abort = 1;
         }
     }

@@ -168,13 +168,14 @@ gemm_umma2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             ptx::prefetch_tensormap(&map_b);
             uint32_t it = 0;
             bool ok = true;
+            int site = 0;
             UmmaWork w;
             for (int wi = 0; ok && umma2_work_item(plan, pair, wi, w); ++wi) {
                 const int tm = w.tm, tn = w.tn;
                 for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
                     const int s = it % C::kStages;
                     const uint32_t ph = (it / C::kStages) & 1;
-                    if (sh->abort || !ptx::mbar_wait(&sh->empty[s], ph ^ 1)) { ok = false; break; }
+                    if (sh->abort || (site = 1, !ptx::mbar_wait(&sh->empty[s], ph ^ 1))) { ok = false; break; }
                     uint8_t* a_dst = ring + s * C::kStageBytes;
                     uint8_t* b_dst = a_dst + C::kABytes;
                     // the leader's "full" barrier of this stage, as seen from this CTA
@@ -188,7 +189,7 @@ gemm_umma2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 }
             }
             if (!ok) {
-                atomicExch(status, kDevTimeout);
+                report_timeout(status, site);
                 sh->abort = 1;
                 // copies already issued must land before the CTA may exit; their bytes are
                 // counted on the leader's barriers, so only the leader can watch them land --
@@ -208,17 +209,18 @@ gemm_umma2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             constexpr uint32_t idesc = ptx::umma_idesc_bf16(C::BM, C::BN, /*a_mn_major=*/false, /*b_mn_major=*/true);
             uint32_t it = 0, tile_it = 0;
             bool ok = true;
+            int site = 0;
             UmmaWork w;
             for (int wi = 0; ok && umma2_work_item(plan, pair, wi, w); ++wi, ++tile_it) {
                 const int a = tile_it & 1;
                 const uint32_t aph = (tile_it >> 1) & 1;
-                if (sh->abort || !ptx::mbar_wait(&sh->tmem_empty[a], aph ^ 1)) { ok = false; break; }
+                if (sh->abort || (site = 2, !ptx::mbar_wait(&sh->tmem_empty[a], aph ^ 1))) { ok = false; break; }
                 ptx::tcgen05_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + a * C::BN;
                 for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
                     const int s = it % C::kStages;
                     const uint32_t ph = (it / C::kStages) & 1;
-                    if (sh->abort || !ptx::mbar_wait(&sh->full[s], ph)) { ok = false; break; }
+                    if (sh->abort || (site = 4, !ptx::mbar_wait(&sh->full[s], ph))) { ok = false; break; }
                     ptx::tcgen05_fence_after_sync();
                     const uint32_t a_addr = ring_base + s * C::kStageBytes;
                     const uint32_t b_addr = a_addr + C::kABytes;
@@ -237,7 +239,7 @@ gemm_umma2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 if (ok) ptx::umma_commit_2cta(&sh->tmem_full[a]);
             }
             if (!ok) {
-                atomicExch(status, kDevTimeout);
+                report_timeout(status, site);
                 sh->abort = 1;
             }
             // nothing may be in flight on the tensor pipe when TMEM is freed
@@ -400,7 +402,7 @@ gemm_umma2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         if (lane == 0) ptx::tma_store_wait_all<0>();
         __syncwarp();
         if (!ok && lane == 0) {
-            atomicExch(status, kDevTimeout);
+            report_timeout(status, 5);
             sh->abort = 1;
         }
     }

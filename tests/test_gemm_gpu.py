@@ -198,7 +198,8 @@ def test_dispatcher_choices(handle):
     assert sel(16, 14336, 4096, BF16) == V.VARIANT_SKINNY_UMMA
     assert sel(4096, 4096, 4096, BF16) == V.VARIANT_UMMA_2CTA
     assert sel(8192, 8192, 16384, BF16) == V.VARIANT_UMMA_2CTA
-    assert sel(128, 4096, 4096, BF16) == V.VARIANT_UMMA
+    assert sel(128, 4096, 4096, BF16) == V.VARIANT_UMMA_2CTA
+    assert sel(64, 4096, 4096, BF16) == V.VARIANT_SKINNY_UMMA and sel(2, 4096, 4096, BF16) == V.VARIANT_SKINNY_UMMA
     assert sel(4096, 4100, 4096, BF16) == V.VARIANT_GENERIC      # N % 8 != 0
     assert sel(0, 1, 1, BF16) == -1
 
