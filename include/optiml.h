@@ -50,7 +50,12 @@ typedef enum {
 
 typedef enum { OPTIML_F32 = 0, OPTIML_BF16 = 1 } optiml_dtype_t;
 
-typedef enum { OPTIML_ACT_NONE = 0, OPTIML_ACT_RELU = 1, OPTIML_ACT_GELU_TANH = 2 } optiml_act_t;
+typedef enum {
+    OPTIML_ACT_NONE = 0,
+    OPTIML_ACT_RELU = 1,      /* max(0, x): Prompts appendix, task 10 */
+    OPTIML_ACT_GELU_TANH = 2, /* tanh form, see the top of this header */
+    OPTIML_ACT_SIGMOID = 3    /* 1 / (1 + exp(-x)): Prompts appendix, task 1 */
+} optiml_act_t;
 
 /* Kernel variants the shape-based dispatcher chooses between. */
 typedef enum {

@@ -23,6 +23,8 @@
  *
  *   GELU_tanh(x) = 0.5 x (1 + tanh( sqrt(2/pi) (x + 0.044715 x^3) ))
  *
+ * act = sigmoid is 1 / (1 + exp(-x)) (Prompts appendix, task 1).
+ *
  * The loop nest is the plain triple loop in i-k-j order (row, reduction index,
  * column) with one fp64 accumulator per output column; rows are dealt to host
  * threads.  No blocking, no vector intrinsics, no reordering of the k sum.
@@ -41,7 +43,7 @@
 #include <string.h>
 
 enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
-enum { ORACLE_ACT_NONE = 0, ORACLE_ACT_RELU = 1, ORACLE_ACT_GELU_TANH = 2 };
+enum { ORACLE_ACT_NONE = 0, ORACLE_ACT_RELU = 1, ORACLE_ACT_GELU_TANH = 2, ORACLE_ACT_SIGMOID = 3 };
 
 /* bf16 is the upper half of an IEEE fp32: widening is a 16-bit shift. */
 double oracle_bf16_to_double(uint16_t bits) {
@@ -93,6 +95,8 @@ double oracle_act(double x, int act) {
         const double c = 0.7978845608028654; /* sqrt(2/pi) */
         return 0.5 * x * (1.0 + tanh(c * (x + 0.044715 * x * x * x)));
     }
+    case ORACLE_ACT_SIGMOID:              /* Prompts appendix, task 1: 1 / (1 + exp(-x)) */
+        return 1.0 / (1.0 + exp(-x));
     default:
         return x;
     }

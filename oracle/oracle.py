@@ -18,6 +18,7 @@ BF16 = 1
 ACT_NONE = 0
 ACT_RELU = 1
 ACT_GELU_TANH = 2
+ACT_SIGMOID = 3
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "gemm_epilogue_oracle.c")

@@ -13,7 +13,7 @@ import os
 import torch
 
 F32, BF16 = 0, 1
-ACT_NONE, ACT_RELU, ACT_GELU_TANH = 0, 1, 2
+ACT_NONE, ACT_RELU, ACT_GELU_TANH, ACT_SIGMOID = 0, 1, 2, 3
 VARIANT_AUTO, VARIANT_GENERIC, VARIANT_F32_TILED, VARIANT_GEMV_SPLITK, VARIANT_SKINNY_UMMA, VARIANT_UMMA = -1, 0, 1, 2, 3, 4
 VARIANT_UMMA_2CTA = 5
 VARIANT_COUNT = 6

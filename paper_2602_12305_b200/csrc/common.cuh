@@ -8,7 +8,7 @@
 
 namespace optiml {
 
-enum : int { kActNone = 0, kActRelu = 1, kActGeluTanh = 2 };
+enum : int { kActNone = 0, kActRelu = 1, kActGeluTanh = 2, kActSigmoid = 3 };
 
 // Device status word values (written by kernels that give up a bounded wait).
 enum : int { kDevOk = 0, kDevTimeout = 7 };
@@ -36,12 +36,20 @@ __device__ __forceinline__ float gelu_tanh(float x) {
     return 0.5f * x * (1.0f + t);
 }
 
+// sigmoid(x) = 1 / (1 + exp(-x)); kFast uses the hardware exponential and reciprocal.
+template <bool kFast>
+__device__ __forceinline__ float sigmoid(float x) {
+    if (kFast) return __fdividef(1.0f, 1.0f + __expf(-x));
+    return 1.0f / (1.0f + expf(-x));
+}
+
 // act(acc + bias) in fp32.  ReLU maps -0 and negatives to +0.
 template <int kAct, bool kFast>
 __device__ __forceinline__ float epilogue(float acc, float bias) {
     float x = acc + bias;
     if (kAct == kActRelu) return x > 0.0f ? x : 0.0f;
     if (kAct == kActGeluTanh) return gelu_tanh<kFast>(x);
+    if (kAct == kActSigmoid) return sigmoid<kFast>(x);
     return x;
 }
 
@@ -51,6 +59,7 @@ __device__ __forceinline__ float epilogue_rt(float acc, float bias, int act) {
     float x = acc + bias;
     if (act == kActRelu) return x > 0.0f ? x : 0.0f;
     if (act == kActGeluTanh) return gelu_tanh<kFast>(x);
+    if (act == kActSigmoid) return sigmoid<kFast>(x);
     return x;
 }
 

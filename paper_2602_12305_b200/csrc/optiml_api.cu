@@ -193,6 +193,9 @@ optiml_status_t launch_f32_cfg(optiml_handle_t h, const float* A, const float* B
     case OPTIML_ACT_GELU_TANH:
         gemm_f32_tiled_kernel<BM, BN, TM, TN, KS, kActGeluTanh><<<(unsigned)tiles, C::kThreads, smem, st>>>(A, B, bias, Y, M, N, K);
         break;
+    case OPTIML_ACT_SIGMOID:
+        gemm_f32_tiled_kernel<BM, BN, TM, TN, KS, kActSigmoid><<<(unsigned)tiles, C::kThreads, smem, st>>>(A, B, bias, Y, M, N, K);
+        break;
     default:
         gemm_f32_tiled_kernel<BM, BN, TM, TN, KS, kActNone><<<(unsigned)tiles, C::kThreads, smem, st>>>(A, B, bias, Y, M, N, K);
         break;
@@ -286,6 +289,10 @@ optiml_status_t launch_umma(optiml_handle_t h, const void* A, const void* B, con
         launch_pdl(gemm_umma_kernel<kActGeluTanh>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
                    plan, h->partials, h->counters, h->status);
         break;
+    case OPTIML_ACT_SIGMOID:
+        launch_pdl(gemm_umma_kernel<kActSigmoid>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
+                   plan, h->partials, h->counters, h->status);
+        break;
     default:
         launch_pdl(gemm_umma_kernel<kActNone>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
                    plan, h->partials, h->counters, h->status);
@@ -316,6 +323,10 @@ optiml_status_t launch_umma2(optiml_handle_t h, const void* A, const void* B, co
         launch_pdl(gemm_umma2_kernel<kActGeluTanh>, grid, dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N,
                    K, plan, h->partials, h->counters, h->status);
         break;
+    case OPTIML_ACT_SIGMOID:
+        launch_pdl(gemm_umma2_kernel<kActSigmoid>, grid, dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N,
+                   K, plan, h->partials, h->counters, h->status);
+        break;
     default:
         launch_pdl(gemm_umma2_kernel<kActNone>, grid, dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
                    plan, h->partials, h->counters, h->status);
@@ -335,9 +346,11 @@ bool configure_kernels() {
     ok &= set_smem(gemm_umma_kernel<kActNone>, UmmaCfg::kSmemBytes);
     ok &= set_smem(gemm_umma_kernel<kActRelu>, UmmaCfg::kSmemBytes);
     ok &= set_smem(gemm_umma_kernel<kActGeluTanh>, UmmaCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma_kernel<kActSigmoid>, UmmaCfg::kSmemBytes);
     ok &= set_smem(gemm_umma2_kernel<kActNone>, Umma2Cfg::kSmemBytes);
     ok &= set_smem(gemm_umma2_kernel<kActRelu>, Umma2Cfg::kSmemBytes);
     ok &= set_smem(gemm_umma2_kernel<kActGeluTanh>, Umma2Cfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2_kernel<kActSigmoid>, Umma2Cfg::kSmemBytes);
     ok &= set_smem(gemm_skinny_umma_kernel<16>, SkinnyCfg<16>::kSmemBytes);
     ok &= set_smem(gemm_skinny_umma_kernel<32>, SkinnyCfg<32>::kSmemBytes);
     ok &= set_smem(gemm_skinny_umma_kernel<64>, SkinnyCfg<64>::kSmemBytes);
@@ -350,7 +363,7 @@ optiml_status_t check_args(optiml_handle_t h, const void* A, const void* B, cons
     if (!h || !A || !B || !Y) return OPTIML_ERR_INVALID_ARG;
     if (M < 1 || N < 1 || K < 1 || M > INT32_MAX || N > INT32_MAX || K > INT32_MAX) return OPTIML_ERR_INVALID_ARG;
     if (dtype != OPTIML_F32 && dtype != OPTIML_BF16) return OPTIML_ERR_INVALID_ARG;
-    if (act != OPTIML_ACT_NONE && act != OPTIML_ACT_RELU && act != OPTIML_ACT_GELU_TANH) return OPTIML_ERR_INVALID_ARG;
+    if (act != OPTIML_ACT_NONE && act != OPTIML_ACT_RELU && act != OPTIML_ACT_GELU_TANH && act != OPTIML_ACT_SIGMOID) return OPTIML_ERR_INVALID_ARG;
     return OPTIML_OK;
 }
 
@@ -575,7 +588,7 @@ extern "C" {
 optiml_status_t optiml_gemv_noalloc(const void* A, const void* B, const void* bias, void* Y, int64_t M, int64_t N,
                                     int64_t K, optiml_act_t act, int device, void* stream) {
     if (!A || !B || !Y || M < 1 || N < 1 || K < 1 || K > INT32_MAX) return OPTIML_ERR_INVALID_ARG;
-    if (act != OPTIML_ACT_NONE && act != OPTIML_ACT_RELU && act != OPTIML_ACT_GELU_TANH) return OPTIML_ERR_INVALID_ARG;
+    if (act != OPTIML_ACT_NONE && act != OPTIML_ACT_RELU && act != OPTIML_ACT_GELU_TANH && act != OPTIML_ACT_SIGMOID) return OPTIML_ERR_INVALID_ARG;
     if (device < 0 || device >= kNoAllocMaxDevices) return OPTIML_ERR_INVALID_ARG;
     // limits of the fixed scratch and of the kernel: refuse, never truncate
     if (M > 4 || N > kNoAllocMaxN || N % 8 != 0) return OPTIML_ERR_UNSUPPORTED;

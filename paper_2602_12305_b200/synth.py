@@ -33,6 +33,7 @@ BF16 = 1
 ACT_NONE = 0
 ACT_RELU = 1
 ACT_GELU_TANH = 2
+ACT_SIGMOID = 3
 
 TENSOR_A = 0
 TENSOR_B = 1

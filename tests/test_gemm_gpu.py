@@ -93,6 +93,16 @@ def test_null_bias_and_act_none(handle):
         parity(handle, c, variant)
 
 
+@pytest.mark.parametrize("variant,name,M,N,K", [(V.VARIANT_GENERIC, "c1", 70, 90, 65), (V.VARIANT_GENERIC, "c4", 70, 90, 65),
+                                                (V.VARIANT_F32_TILED, "c1", 260, 132, 516),
+                                                (V.VARIANT_GEMV_SPLITK, "c2", 1, 1032, 2048),
+                                                (V.VARIANT_SKINNY_UMMA, "c3", 16, 1160, 1096),
+                                                (V.VARIANT_UMMA, "c4", 300, 520, 200),
+                                                (V.VARIANT_UMMA_2CTA, "c4", 300, 520, 1096)])
+def test_sigmoid_epilogue(handle, variant, name, M, N, K):
+    parity(handle, synth.make_case(name, M=M, N=N, K=K, act=synth.ACT_SIGMOID), variant)
+
+
 # ---------------------------------------------------------------- integer-valued inputs: bit-exact
 
 @pytest.mark.parametrize("variant,dtype,M,N,K", [

@@ -158,6 +158,22 @@ def test_gelu_through_the_gemm():
     assert np.abs(y[:, 0] - lib).max() < 1e-15
 
 
+def test_sigmoid_closed_forms_and_library():
+    SIG = oracle.ACT_SIGMOID
+    assert oracle.act(0.0, SIG) == 0.5
+    xs = np.linspace(-12.0, 12.0, 481)
+    s = np.array([oracle.act(x, SIG) for x in xs])
+    sm = np.array([oracle.act(-x, SIG) for x in xs])
+    assert np.allclose(s + sm, 1.0, rtol=0, atol=5e-16)          # sigmoid(x) + sigmoid(-x) = 1
+    assert np.all(np.diff(s) > 0) and 0.0 < s[0] < 1e-5 and 1 - 1e-5 < s[-1] < 1.0
+    assert abs(oracle.act(math.log(3.0), SIG) - 0.75) < 1e-15    # e^x / (1 + e^x) at x = ln 3
+    lib = torch.sigmoid(torch.from_numpy(xs)).numpy()
+    assert np.abs(s - lib).max() < 1e-15
+    # through the GEMM: K = 1, B = [1]
+    y = run(enc(np.array([[-2.0], [0.0], [2.0]]), F32), enc([[1.0]], F32), None, 3, 1, 1, F32, SIG)
+    assert np.abs(y[:, 0] - torch.sigmoid(torch.tensor([-2.0, 0.0, 2.0], dtype=torch.float64)).numpy()).max() < 1e-15
+
+
 # ---------------------------------------------------------------- rounding helpers
 
 def test_bf16_round_ties_to_even():
