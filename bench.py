@@ -394,6 +394,34 @@ def measure(handle, name, args, sampler, device, peaks, peak_src, steps, warmup,
     return out
 
 
+def measure_reductions(handle, device, peaks, peak_src, steps, warmup):
+    """The stand-alone K reductions (sum, dot, MSE) over 2^26 fp32 elements: one pass over HBM."""
+    n = 1 << 26
+    x = torch.from_numpy(synth.uniform(0, 0, n, -1.0, 1.0, synth.F32)).to(device)
+    y = torch.from_numpy(synth.uniform(0, 1, n, -1.0, 1.0, synth.F32)).to(device)
+    out = torch.empty(1, dtype=torch.float32, device=device)
+    stream = torch.cuda.current_stream(device)
+    rows = []
+    for kind, name, nvec in ((0, "sum", 1), (1, "dot", 2), (2, "mse", 2)):
+        for _ in range(warmup):
+            handle.reduce_f32(kind, x, y, out=out, stream=stream)
+        torch.cuda.synchronize(device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            handle.reduce_f32(kind, x, y, out=out, stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize(device)
+        us = e0.elapsed_time(e1) * 1e3 / steps
+        nbytes = 4 * n * nvec + 4
+        gbs = nbytes / 1e9 / (us * 1e-6)
+        rows.append({"kind": name, "n": n, "dtype": "f32", "us_per_step": us, "gbs": gbs,
+                     "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                  "frac": gbs / peaks["hbm_gbs"], "traffic": None, "algorithmic_bytes": nbytes,
+                                  "peak_source": f"of {peak_src}: copy bandwidth"}})
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -450,6 +478,9 @@ def main():
                 "roofline": r["roofline"], "clocks": r["clocks"],
                 "e2e_us": r["e2e_ms"] * 1e3, "gpu_launches": r["launches"]})
 
+    reductions = [] if args.no_per_shape else measure_reductions(handle, device, peaks, peak_src, min(args.steps, 200),
+                                                                 args.warmup)
+
     line = {"metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": region_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32" if case.dtype == synth.F32 else "bf16 inputs, f32 accumulate", "data": "synthetic",
@@ -461,7 +492,7 @@ def main():
                     "d2h_bytes_per_step": main_res["d2h"], "ms_per_step": e2e_ms / main_res["e2e_steps"],
                     "steps": main_res["e2e_steps"]},
             "gpu_launches": main_res["launches"], "replicas": "independent replicas, no data-path collective",
-            "per_shape": per_shape}
+            "per_shape": per_shape, "reductions": reductions}
     sampler.stop()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(case, unit)

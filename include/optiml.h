@@ -164,6 +164,26 @@ optiml_status_t optiml_gemv_noalloc(const void* A, const void* B, const void* bi
  */
 optiml_status_t optiml_get_last_status(optiml_handle_t h);
 
+/*
+ * The K reduction on its own, over fp32 vectors of n elements (paper: Prompts appendix,
+ * task 14 "Reduction": the sum of all elements; task 15 "Dot Product": sum_i x_i * y_i;
+ * task 7 "Mean Square Error": (1/n) sum_i (x_i - y_i)^2 with x the predictions and y the
+ * targets):
+ *
+ *   OPTIML_REDUCE_SUM   *out = sum_i x[i]                       (y is ignored, may be NULL)
+ *   OPTIML_REDUCE_DOT   *out = sum_i x[i] * y[i]
+ *   OPTIML_REDUCE_MSE   *out = (1/n) sum_i (x[i] - y[i])^2
+ *
+ * x, y: device, n fp32 elements, 16-byte aligned, read only, owned by the caller.  out:
+ * device, one fp32, written once.  n >= 1.  One pass over the data; terms are accumulated
+ * in fp32 in many short chains and combined in fp64, in a fixed order.  Enqueued on
+ * `stream`; uses the handle's scratch like the other calls.  Returns INVALID_ARG /
+ * ALIGNMENT before anything is launched, CUDA if the launch failed.
+ */
+typedef enum { OPTIML_REDUCE_SUM = 0, OPTIML_REDUCE_DOT = 1, OPTIML_REDUCE_MSE = 2 } optiml_reduce_t;
+optiml_status_t optiml_reduce_f32(optiml_handle_t h, optiml_reduce_t kind, const float* x, const float* y, int64_t n,
+                                  float* out, void* stream);
+
 /* Force one variant for later calls (tests, profiling), or OPTIML_VARIANT_AUTO to
  * give the choice back to the dispatcher.  A forced variant that cannot run a
  * shape makes optiml_gemm_epilogue return OPTIML_ERR_UNSUPPORTED. */

@@ -18,6 +18,8 @@ VARIANT_AUTO, VARIANT_GENERIC, VARIANT_F32_TILED, VARIANT_GEMV_SPLITK, VARIANT_S
 VARIANT_UMMA_2CTA = 5
 VARIANT_COUNT = 6
 
+REDUCE_SUM, REDUCE_DOT, REDUCE_MSE = 0, 1, 2
+
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ARCH, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(8)
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liboptiml_gemm.so")
@@ -31,6 +33,7 @@ EXPORTS = {
     "optiml_gemm_epilogue_host": (_ci, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _ci, _vp]),
     "optiml_gemv_noalloc": (_ci, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _ci, _vp]),
     "optiml_get_last_status": (_ci, [_vp]),
+    "optiml_reduce_f32": (_ci, [_vp, _ci, _vp, _vp, _i64, _vp, _vp]),
     "optiml_force_variant": (_ci, [_vp, _ci]),
     "optiml_select_variant": (_ci, [_vp, _i64, _i64, _i64, _ci]),
     "optiml_launch_count": (_i64, [_vp]),
@@ -125,7 +128,11 @@ class Handle:
             self._lib.optiml_destroy(self._h)
             self._h = _vp()
 
-    __del__ = destroy
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:      # interpreter shutdown: the library object may already be gone
+            pass
 
     def __enter__(self):
         return self
@@ -178,6 +185,21 @@ class Handle:
                                                    None if bias is None else bias.data_ptr(), Y.data_ptr(), M, N, K,
                                                    dt, act, st), "optiml_gemm_epilogue_host")
         return Y
+
+    def reduce_f32(self, kind: int, x: torch.Tensor, y: torch.Tensor | None = None, out: torch.Tensor | None = None,
+                   stream: torch.cuda.Stream | None = None) -> torch.Tensor:
+        """sum(x), dot(x, y) or mean((x - y)^2) of fp32 CUDA vectors into a one-element fp32 tensor."""
+        for t in (x, y):
+            if t is not None and (not t.is_cuda or t.dtype != torch.float32 or not t.is_contiguous()):
+                raise ValueError("reduce_f32 needs contiguous float32 CUDA tensors")
+        if y is not None and y.numel() != x.numel():
+            raise ValueError("x and y must have the same length")
+        if out is None:
+            out = torch.empty(1, dtype=torch.float32, device=x.device)
+        st = (stream or torch.cuda.current_stream(self.device)).cuda_stream
+        _check(self._lib.optiml_reduce_f32(self._h, int(kind), x.data_ptr(), None if y is None else y.data_ptr(),
+                                           x.numel(), out.data_ptr(), st), "optiml_reduce_f32")
+        return out
 
     def get_last_status(self) -> int:
         return self._lib.optiml_get_last_status(self._h)

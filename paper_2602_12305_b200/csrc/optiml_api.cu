@@ -17,6 +17,7 @@
 #include "kernel_f32.cuh"
 #include "kernel_gemv.cuh"
 #include "kernel_generic.cuh"
+#include "kernel_reduce.cuh"
 #include "kernel_skinny.cuh"
 #include "kernel_umma.cuh"
 #include "kernel_umma2.cuh"
@@ -519,6 +520,37 @@ optiml_status_t optiml_get_last_status(optiml_handle_t h) {
         return OPTIML_ERR_TIMEOUT;
     }
     return OPTIML_OK;
+}
+
+optiml_status_t optiml_reduce_f32(optiml_handle_t h, optiml_reduce_t kind, const float* x, const float* y, int64_t n,
+                                  float* out, void* stream) {
+    if (!h || !x || !out || n < 1) return OPTIML_ERR_INVALID_ARG;
+    if (kind != OPTIML_REDUCE_SUM && kind != OPTIML_REDUCE_DOT && kind != OPTIML_REDUCE_MSE) return OPTIML_ERR_INVALID_ARG;
+    if (kind != OPTIML_REDUCE_SUM && !y) return OPTIML_ERR_INVALID_ARG;
+    if (!aligned16(x) || (kind != OPTIML_REDUCE_SUM && !aligned16(y)) || (reinterpret_cast<uintptr_t>(out) & 3))
+        return OPTIML_ERR_ALIGNMENT;
+    DeviceGuard guard(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // one wave of resident CTAs, fewer when the vector is short: one float4 per thread at least
+    int64_t ctas = (int64_t)h->num_sms * kReduceCtasPerSm;
+    const int64_t need = ceil_div64(ceil_div64(n, 4), kReduceThreads);
+    if (ctas > need) ctas = need;
+    if (ctas < 1) ctas = 1;
+    double* partials = reinterpret_cast<double*>(h->partials);
+    const dim3 grid((unsigned)ctas), block(kReduceThreads);
+    switch (kind) {
+    case OPTIML_REDUCE_DOT:
+        launch_pdl(reduce_f32_kernel<kReduceDot>, grid, block, 0, st, x, y, n, out, partials, h->counters);
+        break;
+    case OPTIML_REDUCE_MSE:
+        launch_pdl(reduce_f32_kernel<kReduceMse>, grid, block, 0, st, x, y, n, out, partials, h->counters);
+        break;
+    default:
+        launch_pdl(reduce_f32_kernel<kReduceSum>, grid, block, 0, st, x, y, n, out, partials, h->counters);
+        break;
+    }
+    h->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
 }
 
 optiml_status_t optiml_force_variant(optiml_handle_t h, optiml_variant_t v) {
