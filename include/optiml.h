@@ -62,7 +62,7 @@ typedef enum {
     OPTIML_VARIANT_AUTO = -1,
     OPTIML_VARIANT_GENERIC = 0,     /* predicated FMA tiles: any shape, any alignment, both dtypes      */
     OPTIML_VARIANT_F32_TILED = 1,   /* fp32 FMA tiles, 128-bit loads: needs N % 4 == 0 and K % 4 == 0    */
-    OPTIML_VARIANT_GEMV_SPLITK = 2, /* bf16, M <= 4: split-K streaming with 128-bit loads, N % 8 == 0    */
+    OPTIML_VARIANT_GEMV_SPLITK = 2, /* M <= 4: split-K streaming, 128-bit loads; N % 8 (bf16) / 4 (fp32) */
     OPTIML_VARIANT_SKINNY_UMMA = 3, /* bf16, M <= 128: stream-K over B with tcgen05 (N is the MMA M dim) */
     OPTIML_VARIANT_UMMA = 4,        /* bf16: persistent TMA + tcgen05 + TMEM tiles, N % 8 == K % 8 == 0  */
     OPTIML_VARIANT_UMMA_2CTA = 5,   /* bf16: the same with CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles) */

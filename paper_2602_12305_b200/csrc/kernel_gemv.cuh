@@ -1,8 +1,8 @@
-// GEMV / very skinny variant (bf16, M <= 4): the problem is a stream over B, so the
-// kernel is organised around HBM: every lane issues 128-bit non-allocating loads of B
-// (8 bf16 columns), a warp covers one 512-byte row segment per load, eight warps take
-// interleaved rows, and kGemvUnroll independent loads per thread are in flight before the
-// first FMA.  K is split across gridDim.y CTAs so that the grid fills every SM once
+// GEMV / very skinny variant (M <= 4; bf16 or fp32): the problem is a stream over B, so
+// the kernel is organised around HBM: every lane issues 128-bit non-allocating loads of B
+// (8 bf16 or 4 fp32 columns), a warp covers one 512-byte row segment per load, eight warps
+// take interleaved rows, and kGemvUnroll independent loads per thread are in flight before
+// the first FMA.  K is split across gridDim.y CTAs so that the grid fills every SM once
 // (gemv_ctas_per_sm CTAs per SM).
 //
 // Reduction of the K slices: warps -> shared memory (fixed order) -> CTA partial in the
@@ -16,42 +16,60 @@
 
 namespace optiml {
 
-constexpr int kGemvCols = 256;     // columns per CTA: 32 lanes x 8 bf16
 constexpr int kGemvWarps = 8;
 constexpr int kGemvThreads = kGemvWarps * 32;
-// Measured on B200 (1 x 8192 x 8192): many resident warps with few loads each beat few
+// Measured on B200 (1 x 8192 x 8192 bf16): many resident warps with few loads each beat few
 // warps with deep unrolling -- 4 loads in flight per thread and 5 CTAs per SM (40 warps)
 // stream at 5.5 TB/s, 8 loads and 2 CTAs at 4.5 TB/s.
 constexpr int kGemvUnroll = 4;
 // resident CTAs per SM: M = 1 needs few registers; 2-4 rows of A need more accumulators
 constexpr int gemv_ctas_per_sm(int mr) { return mr == 1 ? 5 : 2; }
 
-template <int MR>
+// columns per 16-byte load and per CTA (32 lanes)
+template <typename T> struct GemvVec { static constexpr int V = 16 / (int)sizeof(T); static constexpr int kCols = 32 * V; };
+constexpr int kGemvCols = GemvVec<__nv_bfloat16>::kCols;       // 256 (bf16); fp32: 128
+
+__device__ __forceinline__ void gemv_unpack(const uint4& v, float (&b)[8], __nv_bfloat16) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        b[2 * q] = bf16lo_to_f32(w[q]);
+        b[2 * q + 1] = bf16hi_to_f32(w[q]);
+    }
+}
+__device__ __forceinline__ void gemv_unpack(const uint4& v, float (&b)[4], float) {
+    b[0] = __uint_as_float(v.x);
+    b[1] = __uint_as_float(v.y);
+    b[2] = __uint_as_float(v.z);
+    b[3] = __uint_as_float(v.w);
+}
+
+template <typename T, int MR>
 __global__ void __launch_bounds__(kGemvThreads, gemv_ctas_per_sm(MR))
-gemv_splitk_kernel(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __restrict__ B,
-                   const __nv_bfloat16* __restrict__ bias, __nv_bfloat16* __restrict__ Y,
+gemv_splitk_kernel(const T* __restrict__ A, const T* __restrict__ B, const T* __restrict__ bias, T* __restrict__ Y,
                    int M, int N, int K, int act, float* __restrict__ partials, unsigned int* __restrict__ counters) {
-    __shared__ float red[kGemvWarps][MR][kGemvCols];
+    constexpr int V = GemvVec<T>::V, kCols = GemvVec<T>::kCols;
+    __shared__ float red[kGemvWarps][MR][kCols];
     __shared__ int s_last;
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int cb = blockIdx.x, slice = blockIdx.y, S = gridDim.y;
-    const int64_t n = (int64_t)cb * kGemvCols + lane * 8;
-    const bool n_ok = n < N;                                   // N % 8 == 0: all 8 columns or none
+    const int64_t n = (int64_t)cb * kCols + lane * V;
+    const bool n_ok = n < N;                                   // N % V == 0: all V columns or none
     const int k_begin = (int)((int64_t)K * slice / S);
     const int k_end = (int)((int64_t)K * (slice + 1) / S);
 
-    float acc[MR][8];
+    float acc[MR][V];
 #pragma unroll
     for (int m = 0; m < MR; ++m)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[m][j] = 0.0f;
+        for (int j = 0; j < V; ++j) acc[m][j] = 0.0f;
 
     // launched as a programmatic dependent: wait for the previous kernel before touching memory
     ptx::griddep_wait();
     ptx::griddep_launch_dependents();
 
-    const __nv_bfloat16* bp = B + n;
+    const T* bp = B + n;
     for (int kb = k_begin + warp; kb < k_end; kb += kGemvWarps * kGemvUnroll) {
         uint4 v[kGemvUnroll];
         float a[kGemvUnroll][MR];
@@ -61,21 +79,16 @@ gemv_splitk_kernel(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __r
             const bool ok = n_ok && k < k_end;
             v[u] = ok ? ld_stream_v4(bp + (int64_t)k * N) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-            for (int m = 0; m < MR; ++m)
-                a[u][m] = (k < k_end && m < M) ? __bfloat162float(A[(int64_t)m * K + k]) : 0.0f;
+            for (int m = 0; m < MR; ++m) a[u][m] = (k < k_end && m < M) ? to_f32(A[(int64_t)m * K + k]) : 0.0f;
         }
 #pragma unroll
         for (int u = 0; u < kGemvUnroll; ++u) {
-            const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+            float b[V];
+            gemv_unpack(v[u], b, T());
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const float b0 = bf16lo_to_f32(w[q]), b1 = bf16hi_to_f32(w[q]);
+            for (int j = 0; j < V; ++j)
 #pragma unroll
-                for (int m = 0; m < MR; ++m) {
-                    acc[m][2 * q] = fmaf(a[u][m], b0, acc[m][2 * q]);
-                    acc[m][2 * q + 1] = fmaf(a[u][m], b1, acc[m][2 * q + 1]);
-                }
-            }
+                for (int m = 0; m < MR; ++m) acc[m][j] = fmaf(a[u][m], b[j], acc[m][j]);
         }
     }
 
@@ -83,24 +96,29 @@ gemv_splitk_kernel(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __r
 #pragma unroll
     for (int m = 0; m < MR; ++m)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) red[warp][m][lane * 8 + j] = acc[m][j];
+        for (int j = 0; j < V; ++j) red[warp][m][lane * V + j] = acc[m][j];
     __syncthreads();
 
     const int t = threadIdx.x;                 // one output column per thread from here on
-    const int64_t col = (int64_t)cb * kGemvCols + t;
+    const bool has_col = t < kCols;            // fp32: the upper half of the CTA has no column
+    const int64_t col = (int64_t)cb * kCols + t;
     float sum[MR];
 #pragma unroll
     for (int m = 0; m < MR; ++m) {
         float s = 0.0f;
+        if (has_col) {
 #pragma unroll
-        for (int w = 0; w < kGemvWarps; ++w) s += red[w][m][t];
+            for (int w = 0; w < kGemvWarps; ++w) s += red[w][m][t];
+        }
         sum[m] = s;
     }
 
     if (S > 1) {
-        float* mine = partials + ((size_t)cb * S + slice) * (MR * kGemvCols);
+        float* mine = partials + ((size_t)cb * S + slice) * (MR * kCols);
+        if (has_col) {
 #pragma unroll
-        for (int m = 0; m < MR; ++m) mine[m * kGemvCols + t] = sum[m];
+            for (int m = 0; m < MR; ++m) mine[m * kCols + t] = sum[m];
+        }
         __threadfence();
         __syncthreads();
         if (t == 0) {
@@ -110,30 +128,36 @@ gemv_splitk_kernel(const __nv_bfloat16* __restrict__ A, const __nv_bfloat16* __r
         __syncthreads();
         if (!s_last) return;
         __threadfence();
-        const float* all = partials + (size_t)cb * S * (MR * kGemvCols);
+        const float* all = partials + (size_t)cb * S * (MR * kCols);
         // slices in order, eight loads in flight at a time (one dependent chain of L2 round
         // trips per slice would cost more than the whole stream over B)
+        if (has_col) {
 #pragma unroll
-        for (int m = 0; m < MR; ++m) {
-            float s = 0.0f;
-            for (int q0 = 0; q0 < S; q0 += 8) {
-                float v[8];
+            for (int m = 0; m < MR; ++m) {
+                float s = 0.0f;
+                for (int q0 = 0; q0 < S; q0 += 8) {
+                    float v[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    v[i] = (q0 + i < S) ? __ldcg(all + (size_t)(q0 + i) * (MR * kGemvCols) + m * kGemvCols + t) : 0.0f;
+                    for (int i = 0; i < 8; ++i)
+                        v[i] = (q0 + i < S) ? __ldcg(all + (size_t)(q0 + i) * (MR * kCols) + m * kCols + t) : 0.0f;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) s += v[i];
+                    for (int i = 0; i < 8; ++i) s += v[i];
+                }
+                sum[m] = s;
             }
-            sum[m] = s;
         }
         if (t == 0) counters[cb] = 0u;         // ready for the next call on this stream
     }
 
-    if (col < N) {
-        const float bv = bias ? __bfloat162float(bias[col]) : 0.0f;
+    if (has_col && col < N) {
+        const float bv = bias ? to_f32(bias[col]) : 0.0f;
 #pragma unroll
-        for (int m = 0; m < MR; ++m)
-            if (m < M) Y[(int64_t)m * N + col] = __float2bfloat16_rn(epilogue_rt<true>(sum[m], bv, act));
+        for (int m = 0; m < MR; ++m) {
+            if (m >= M) continue;
+            // tanhf / expf for fp32 output, the hardware approximations for bf16 output
+            const float y = sizeof(T) == 4 ? epilogue_rt<false>(sum[m], bv, act) : epilogue_rt<true>(sum[m], bv, act);
+            Y[(int64_t)m * N + col] = from_f32<T>(y);
+        }
     }
 }
 

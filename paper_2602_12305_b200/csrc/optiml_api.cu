@@ -117,7 +117,8 @@ bool variant_supports(int v, int64_t M, int64_t N, int64_t K, int dtype, bool al
     case OPTIML_VARIANT_F32_TILED:
         return dtype == OPTIML_F32 && N % 4 == 0 && K % 4 == 0 && al16;
     case OPTIML_VARIANT_GEMV_SPLITK:
-        return dtype == OPTIML_BF16 && M <= 4 && N % 8 == 0 && al16 && ceil_div64(N, kGemvCols) <= kNumCounters;
+        return M <= 4 && N % (dtype == OPTIML_F32 ? 4 : 8) == 0 && al16 &&
+               ceil_div64(N, dtype == OPTIML_F32 ? GemvVec<float>::kCols : kGemvCols) <= kNumCounters;
     case OPTIML_VARIANT_SKINNY_UMMA:
         return dtype == OPTIML_BF16 && M <= 128 && N % 8 == 0 && K % 8 == 0 && al16 &&
                ceil_div64(N, 128) <= kNumCounters;
@@ -137,9 +138,13 @@ bool variant_supports(int v, int64_t M, int64_t N, int64_t K, int dtype, bool al
 // (stream-K tcgen05 with N as the MMA M dimension), larger M is compute-bound.
 int choose_variant(optiml_handle_t h, int64_t M, int64_t N, int64_t K, int dtype, bool al16) {
     if (h->forced != OPTIML_VARIANT_AUTO) return h->forced;
-    if (dtype == OPTIML_F32)
+    if (dtype == OPTIML_F32) {
+        // fp32 has no tensor-core path: up to 4 rows stream over B (measured 1 x 8192 x 8192: 163 us
+        // on the tiles, a fifth of that on the streaming kernel), everything else goes to the FMA tiles
+        if (M <= 4 && variant_supports(OPTIML_VARIANT_GEMV_SPLITK, M, N, K, dtype, al16)) return OPTIML_VARIANT_GEMV_SPLITK;
         return variant_supports(OPTIML_VARIANT_F32_TILED, M, N, K, dtype, al16) ? OPTIML_VARIANT_F32_TILED
                                                                                  : OPTIML_VARIANT_GENERIC;
+    }
     if (M == 1 && variant_supports(OPTIML_VARIANT_GEMV_SPLITK, M, N, K, dtype, al16)) return OPTIML_VARIANT_GEMV_SPLITK;
     if (M <= 64 && variant_supports(OPTIML_VARIANT_SKINNY_UMMA, M, N, K, dtype, al16)) return OPTIML_VARIANT_SKINNY_UMMA;
     // above 64 rows a CTA pair shares one 256 x 256 tile (a third less operand traffic per flop); measured
@@ -221,26 +226,40 @@ optiml_status_t launch_f32(optiml_handle_t h, const void* A, const void* B, cons
 template <int MR>
 void launch_gemv_mr(const void* A, const void* B, const void* bias, void* Y, int M, int N, int K, int act, dim3 grid,
                     float* partials, unsigned int* counters, cudaStream_t st) {
-    launch_pdl(gemv_splitk_kernel<MR>, grid, dim3(kGemvThreads), 0, st, (const __nv_bfloat16*)A,
+    launch_pdl(gemv_splitk_kernel<__nv_bfloat16, MR>, grid, dim3(kGemvThreads), 0, st, (const __nv_bfloat16*)A,
                (const __nv_bfloat16*)B, (const __nv_bfloat16*)bias, (__nv_bfloat16*)Y, M, N, K, act, partials, counters);
 }
 
+template <int MR>
+void launch_gemv_f32_mr(const void* A, const void* B, const void* bias, void* Y, int M, int N, int K, int act, dim3 grid,
+                        float* partials, unsigned int* counters, cudaStream_t st) {
+    launch_pdl(gemv_splitk_kernel<float, MR>, grid, dim3(kGemvThreads), 0, st, (const float*)A, (const float*)B,
+               (const float*)bias, (float*)Y, M, N, K, act, partials, counters);
+}
+
 optiml_status_t launch_gemv(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
-                            int K, int act, cudaStream_t st) {
+                            int K, int dtype, int act, cudaStream_t st) {
     const int MR = M == 1 ? 1 : (M == 2 ? 2 : 4);
-    const int64_t col_blocks = ceil_div64(N, kGemvCols);
+    const int cols = dtype == OPTIML_F32 ? GemvVec<float>::kCols : GemvVec<__nv_bfloat16>::kCols;
+    const int64_t col_blocks = ceil_div64(N, cols);
     // K slices: fill every SM with its resident CTAs in one wave, keep at least 64 rows per slice,
     // stay inside the scratch and the 65535 limit of gridDim.y.
     int64_t S = (gemv_ctas_per_sm(MR) * (int64_t)h->num_sms) / col_blocks;
     if (S > K / 64) S = K / 64;
-    const int64_t per_slice = (int64_t)MR * kGemvCols * sizeof(float);
+    const int64_t per_slice = (int64_t)MR * cols * sizeof(float);
     if (S * col_blocks * per_slice > (int64_t)kPartialBytes) S = kPartialBytes / (col_blocks * per_slice);
     if (S > 65535) S = 65535;
     if (S < 1) S = 1;
     dim3 grid((unsigned)col_blocks, (unsigned)S);
-    if (MR == 1) launch_gemv_mr<1>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
-    else if (MR == 2) launch_gemv_mr<2>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
-    else launch_gemv_mr<4>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
+    if (dtype == OPTIML_F32) {
+        if (MR == 1) launch_gemv_f32_mr<1>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
+        else if (MR == 2) launch_gemv_f32_mr<2>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
+        else launch_gemv_f32_mr<4>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
+    } else {
+        if (MR == 1) launch_gemv_mr<1>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
+        else if (MR == 2) launch_gemv_mr<2>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
+        else launch_gemv_mr<4>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
+    }
     h->launches += 1;
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
 }
@@ -458,7 +477,7 @@ optiml_status_t optiml_gemm_epilogue(optiml_handle_t h, const void* A, const voi
     case OPTIML_VARIANT_F32_TILED:
         return launch_f32(h, A, B, bias, Y, m, n, k, (int)act, st);
     case OPTIML_VARIANT_GEMV_SPLITK:
-        return launch_gemv(h, A, B, bias, Y, m, n, k, (int)act, st);
+        return launch_gemv(h, A, B, bias, Y, m, n, k, (int)dtype, (int)act, st);
     case OPTIML_VARIANT_SKINNY_UMMA:
         return launch_skinny(h, A, B, bias, Y, m, n, k, (int)act, st);
     case OPTIML_VARIANT_UMMA:

@@ -63,6 +63,15 @@ def test_gemv_variant(handle, M, N, K, act):
     parity(handle, synth.make_case("c2", M=M, N=N, K=K, act=act), V.VARIANT_GEMV_SPLITK)
 
 
+@pytest.mark.parametrize("M,N,K", [(1, 512, 1024), (1, 132, 100), (2, 1028, 333), (3, 516, 777), (4, 4096, 300),
+                                   (1, 4, 1), (1, 8192, 8192)])
+@pytest.mark.parametrize("act", [RELU, GELU])
+def test_gemv_variant_fp32(handle, M, N, K, act):
+    c = synth.make_case("c1", M=M, N=N, K=K, act=act)
+    assert handle.select_variant(M, N, K, F32) == V.VARIANT_GEMV_SPLITK
+    parity(handle, c, V.VARIANT_GEMV_SPLITK)
+
+
 @pytest.mark.parametrize("M,N,K", [(16, 1160, 1096),     # 180 units over 148 CTAs: tiles split mid-K
                                    (16, 20480, 64),      # one K block per tile: every segment whole
                                    (1, 1024, 2048), (5, 136, 8), (17, 392, 520), (33, 1288, 264), (64, 2056, 712),
@@ -108,6 +117,7 @@ def test_sigmoid_epilogue(handle, variant, name, M, N, K):
 @pytest.mark.parametrize("variant,dtype,M,N,K", [
     (V.VARIANT_GENERIC, F32, 70, 90, 300), (V.VARIANT_GENERIC, BF16, 70, 90, 300),
     (V.VARIANT_F32_TILED, F32, 96, 160, 512), (V.VARIANT_GEMV_SPLITK, BF16, 1, 1024, 4096),
+    (V.VARIANT_GEMV_SPLITK, F32, 1, 1028, 4096), (V.VARIANT_GEMV_SPLITK, F32, 3, 260, 1000),
     (V.VARIANT_GEMV_SPLITK, BF16, 4, 520, 1000), (V.VARIANT_SKINNY_UMMA, BF16, 16, 1160, 1096),
     (V.VARIANT_SKINNY_UMMA, BF16, 48, 648, 2048), (V.VARIANT_UMMA, BF16, 384, 776, 1024),
     (V.VARIANT_UMMA_2CTA, BF16, 384, 776, 1024), (V.VARIANT_UMMA_2CTA, BF16, 1000, 520, 320)])
