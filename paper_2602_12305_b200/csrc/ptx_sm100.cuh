@@ -47,20 +47,22 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
     return t;
 }
 
-// Wait for the phase with the given parity to complete, but never forever: the wall
-// clock is checked every 64 failed polls and after kWaitLimitNs (two seconds, far
-// beyond any legitimate wait in these kernels) the wait gives up and returns false.
-// The caller then records a time-out in the handle's status word and leaves through
-// the common tear-down path.
-constexpr uint64_t kWaitLimitNs = 2000000000ull;
+// Wait for the phase with the given parity to complete, but never forever: the SM's cycle
+// counter is checked every 64 failed polls and after kWaitLimitCycles (two to three seconds
+// at 1.3-1.97 GHz, far beyond any legitimate wait in these kernels) the wait gives up and
+// returns false.  The caller then records a time-out in the handle's status word and leaves
+// through the common tear-down path.  (The cycle counter, not %globaltimer: the global timer
+// can be stepped from outside, while clock64 only ever counts this SM's cycles.  With the
+// global timer one time-out was reported in some 50 000 launches and never reproduced.)
+constexpr long long kWaitLimitCycles = 4000000000ll;
 
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_timer_ns();
+    const long long t0 = clock64();
     for (uint32_t i = 1;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 63u) == 0u) {
-            if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+            if (clock64() - t0 > kWaitLimitCycles) return false;
             __nanosleep(32);
         }
     }
