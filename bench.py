@@ -47,7 +47,8 @@ FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel,
 # from the ncu captures summarised under profiles/; None = not captured for the current kernel.
-NCU_TRAFFIC_BYTES = {"c1": 542208, "c2": 137838336, "c3": 121811968, "c4": 110100992, "c5": 2564892440}
+NCU_TRAFFIC_BYTES = {"c1": 542464, "c2": 137573632, "c3": 121340928, "c4": 108860672, "c5": 2799265680,
+                     "sum": 272239616, "dot": 540065280, "mse": None}
 
 
 def load_peaks():
@@ -423,7 +424,7 @@ def measure_reductions(handle, device, peaks, peak_src, steps, warmup):
         gbs = nbytes / 1e9 / (us * 1e-6)
         rows.append({"kind": name, "n": n, "dtype": "f32", "us_per_step": us, "gbs": gbs,
                      "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                  "frac": gbs / peaks["hbm_gbs"], "traffic": None, "algorithmic_bytes": nbytes,
+                                  "frac": gbs / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(name), "algorithmic_bytes": nbytes,
                                   "peak_source": f"of {peak_src}: copy bandwidth"}})
     return rows
 

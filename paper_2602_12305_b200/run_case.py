@@ -1,8 +1,9 @@
 """Run one named workload a few times through the C ABI -- the command line used for
 profiling (ncu) and for quick timing of a forced variant.
 
-    python -m paper_2602_12305_b200.run_case --workload c3 [--variant auto|0..4] [--iters 3]
+    python -m paper_2602_12305_b200.run_case --workload c3 [--variant auto|0..5] [--iters 3]
         [--M m --N n --K k] [--sets 2] [--time]
+    python -m paper_2602_12305_b200.run_case --reduce sum|dot|mse [--n 67108864] [--iters 3]
 
 Each iteration uses the next of `--sets` distinct buffer sets.  With --time, CUDA-event
 times per launch are printed (median / min) with the implied TFLOP/s and GB/s.
@@ -24,6 +25,30 @@ def _dev(arr, dtype, shape):
     return torch.from_numpy(arr.view(np.int16)).view(torch.bfloat16).view(*shape).cuda()
 
 
+def run_reduce(a):
+    kind = {"sum": binding.REDUCE_SUM, "dot": binding.REDUCE_DOT, "mse": binding.REDUCE_MSE}[a.reduce]
+    h = binding.Handle(0)
+    x = torch.from_numpy(synth.uniform(0, 0, a.n, -1.0, 1.0, synth.F32)).cuda()
+    y = torch.from_numpy(synth.uniform(0, 1, a.n, -1.0, 1.0, synth.F32)).cuda()
+    out = torch.empty(1, dtype=torch.float32, device="cuda")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(a.warmup):
+        h.reduce_f32(kind, x, y, out=out)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(a.iters):
+        h.reduce_f32(kind, x, y, out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    status = h.get_last_status()
+    us = e0.elapsed_time(e1) * 1e3 / a.iters
+    nbytes = 4 * a.n * (1 if a.reduce == "sum" else 2) + 4
+    print(f"reduce {a.reduce} n={a.n}: {a.iters} launches, result {out.item():.9g}, status {binding.status_string(status)}, "
+          f"{us:.2f} us per launch, {nbytes / 1e3 / us:.0f} GB/s")
+    h.destroy()
+    return 0 if status == binding.OK else 1
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="c2", choices=sorted(synth.WORKLOADS))
@@ -36,7 +61,11 @@ def main():
     ap.add_argument("--K", type=int)
     ap.add_argument("--time", action="store_true")
     ap.add_argument("--no-step-events", action="store_true", help="one event pair around all launches only")
+    ap.add_argument("--reduce", choices=["sum", "dot", "mse"], help="run the stand-alone reduction instead")
+    ap.add_argument("--n", type=int, default=1 << 26, help="vector length for --reduce")
     a = ap.parse_args()
+    if a.reduce:
+        return run_reduce(a)
 
     c = synth.make_case(a.workload, M=a.M, N=a.N, K=a.K)
     h = binding.Handle(0)
