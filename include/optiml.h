@@ -184,6 +184,33 @@ typedef enum { OPTIML_REDUCE_SUM = 0, OPTIML_REDUCE_DOT = 1, OPTIML_REDUCE_MSE =
 optiml_status_t optiml_reduce_f32(optiml_handle_t h, optiml_reduce_t kind, const float* x, const float* y, int64_t n,
                                   float* out, void* stream);
 
+/*
+ * Multi-head self-attention (paper: Prompts appendix, task 6).  Q, K, V and Y are N x d_model,
+ * dense row-major; with d_k = d_model / heads, head i owns columns [i d_k, (i+1) d_k) of each:
+ *
+ *   head_i = softmax(Q_i K_i^T / sqrt(d_k)) V_i     softmax over the keys, row by row
+ *   Y      = Concat(head_1, ..., head_h)             head i written back to its own columns
+ *
+ * No mask, no projection.  Q, K, V: device, N * d_model elements of dtype, read only.  Y: device,
+ * N * d_model elements of dtype, written once, must not overlap the inputs.  N >= 1, d_model a
+ * multiple of heads.  The caller owns all four buffers; they must stay valid until the work has
+ * run.  Inputs must be finite.
+ *
+ * Arithmetic.  OPTIML_BF16 with d_k = 64 or 128, 16-byte aligned pointers and d_model % 8 == 0
+ * runs on the tensor cores: exact bf16 products, fp32 accumulation, softmax in fp32 with
+ * exp2 on the special-function unit, probabilities rounded to bf16 before they multiply V,
+ * their sum kept unrounded in fp32, one rounding of the quotient to bf16 at the store.  Any other
+ * d_k <= 256, unaligned pointers and OPTIML_F32 run on a plain FMA kernel (fp32 throughout; bf16
+ * rounded once at the store).  d_k > 256 returns OPTIML_ERR_UNSUPPORTED.  A forced
+ * OPTIML_VARIANT_GENERIC (optiml_force_variant) selects the FMA kernel; any other forced variant
+ * demands the tensor-core kernel and returns UNSUPPORTED where it cannot run.
+ *
+ * Enqueued on `stream`; INVALID_ARG / ALIGNMENT / UNSUPPORTED before anything is launched, CUDA if
+ * the launch failed; a device-side time-out is reported by optiml_get_last_status.
+ */
+optiml_status_t optiml_mhsa(optiml_handle_t h, const void* Q, const void* K, const void* V, void* Y, int64_t N,
+                            int64_t d_model, int64_t heads, optiml_dtype_t dtype, void* stream);
+
 /* Force one variant for later calls (tests, profiling), or OPTIML_VARIANT_AUTO to
  * give the choice back to the dispatcher.  A forced variant that cannot run a
  * shape makes optiml_gemm_epilogue return OPTIML_ERR_UNSUPPORTED. */

@@ -34,6 +34,7 @@ EXPORTS = {
     "optiml_gemv_noalloc": (_ci, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _ci, _vp]),
     "optiml_get_last_status": (_ci, [_vp]),
     "optiml_reduce_f32": (_ci, [_vp, _ci, _vp, _vp, _i64, _vp, _vp]),
+    "optiml_mhsa": (_ci, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _vp]),
     "optiml_force_variant": (_ci, [_vp, _ci]),
     "optiml_select_variant": (_ci, [_vp, _i64, _i64, _i64, _ci]),
     "optiml_launch_count": (_i64, [_vp]),
@@ -200,6 +201,22 @@ class Handle:
         _check(self._lib.optiml_reduce_f32(self._h, int(kind), x.data_ptr(), None if y is None else y.data_ptr(),
                                            x.numel(), out.data_ptr(), st), "optiml_reduce_f32")
         return out
+
+    def mhsa(self, Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, heads: int, Y: torch.Tensor | None = None,
+             stream: torch.cuda.Stream | None = None) -> torch.Tensor:
+        """Multi-head self-attention of (N, d_model) CUDA tensors (float32 or bfloat16), heads in column blocks."""
+        n, d_model = Q.shape
+        for t in (Q, K, V):
+            if not t.is_cuda or t.dtype != Q.dtype or tuple(t.shape) != (n, d_model) or not t.is_contiguous():
+                raise ValueError("mhsa needs contiguous CUDA tensors of one dtype and shape (N, d_model)")
+        if Q.dtype not in (torch.float32, torch.bfloat16):
+            raise ValueError("mhsa supports float32 and bfloat16")
+        if Y is None:
+            Y = torch.empty_like(Q)
+        st = (stream or torch.cuda.current_stream(self.device)).cuda_stream
+        _check(self._lib.optiml_mhsa(self._h, Q.data_ptr(), K.data_ptr(), V.data_ptr(), Y.data_ptr(), n, d_model, int(heads),
+                                     F32 if Q.dtype == torch.float32 else BF16, st), "optiml_mhsa")
+        return Y
 
     def get_last_status(self) -> int:
         return self._lib.optiml_get_last_status(self._h)

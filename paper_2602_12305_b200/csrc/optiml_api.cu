@@ -7,6 +7,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -17,6 +18,7 @@
 #include "kernel_f32.cuh"
 #include "kernel_gemv.cuh"
 #include "kernel_generic.cuh"
+#include "kernel_mhsa.cuh"
 #include "kernel_reduce.cuh"
 #include "kernel_skinny.cuh"
 #include "kernel_umma.cuh"
@@ -375,7 +377,42 @@ bool configure_kernels() {
     ok &= set_smem(gemm_skinny_umma_kernel<32>, SkinnyCfg<32>::kSmemBytes);
     ok &= set_smem(gemm_skinny_umma_kernel<64>, SkinnyCfg<64>::kSmemBytes);
     ok &= set_smem(gemm_skinny_umma_kernel<128>, SkinnyCfg<128>::kSmemBytes);
+    ok &= set_smem(mhsa_umma_kernel<64>, MhsaCfg<64>::kSmemBytes);
+    ok &= set_smem(mhsa_umma_kernel<128>, MhsaCfg<128>::kSmemBytes);
     return ok;
+}
+
+template <int DK>
+optiml_status_t launch_mhsa_umma(optiml_handle_t h, const void* Q, const void* K, const void* V, void* Y, int N,
+                                 int d_model, int heads, cudaStream_t st) {
+    using C = MhsaCfg<DK>;
+    const CUtensorMap* mq = get_map(h, Q, (uint64_t)N, (uint64_t)d_model, 128, 64);
+    const CUtensorMap* mk = get_map(h, K, (uint64_t)N, (uint64_t)d_model, 128, 64);
+    const CUtensorMap* mv = get_map(h, V, (uint64_t)N, (uint64_t)d_model, 128, 64);
+    if (!mq || !mk || !mv) return OPTIML_ERR_CUDA;
+    const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)DK));
+    const dim3 grid((unsigned)ceil_div64(N, C::kQTiles * C::BQ), (unsigned)heads);
+    launch_pdl(mhsa_umma_kernel<DK>, grid, dim3(C::kThreads), C::kSmemBytes, st, *mq, *mk, *mv, (__nv_bfloat16*)Y, N,
+               d_model, scale_log2, h->status);
+    h->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+template <typename T>
+optiml_status_t launch_mhsa_generic(optiml_handle_t h, const void* Q, const void* K, const void* V, void* Y, int N,
+                                    int d_model, int heads, cudaStream_t st) {
+    const int64_t warps = (int64_t)N * heads;
+    const float scale = (float)(1.0 / sqrt((double)(d_model / heads)));
+    launch_pdl(mhsa_generic_kernel<T>, dim3((unsigned)ceil_div64(warps, kMhsaGenericWarps)), dim3(kMhsaGenericWarps * 32), 0,
+               st, (const T*)Q, (const T*)K, (const T*)V, (T*)Y, N, d_model, heads, scale);
+    h->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+// tcgen05 attention needs bf16, d_k of 64 or 128 and 16-byte aligned rows
+bool mhsa_umma_supported(int64_t d_model, int64_t heads, int dtype, bool al16) {
+    const int64_t dk = d_model / heads;
+    return dtype == OPTIML_BF16 && (dk == 64 || dk == 128) && al16 && heads <= 65535;
 }
 
 optiml_status_t check_args(optiml_handle_t h, const void* A, const void* B, const void* Y, int64_t M, int64_t N,
@@ -570,6 +607,34 @@ optiml_status_t optiml_reduce_f32(optiml_handle_t h, optiml_reduce_t kind, const
     }
     h->launches += 1;
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+optiml_status_t optiml_mhsa(optiml_handle_t h, const void* Q, const void* K, const void* V, void* Y, int64_t N,
+                            int64_t d_model, int64_t heads, optiml_dtype_t dtype, void* stream) {
+    if (!h || !Q || !K || !V || !Y) return OPTIML_ERR_INVALID_ARG;
+    if (N < 1 || d_model < 1 || heads < 1 || N > INT32_MAX || d_model > INT32_MAX || d_model % heads != 0)
+        return OPTIML_ERR_INVALID_ARG;
+    if (dtype != OPTIML_F32 && dtype != OPTIML_BF16) return OPTIML_ERR_INVALID_ARG;
+    const uintptr_t es = dtype == OPTIML_F32 ? 4 : 2;
+    const uintptr_t all = reinterpret_cast<uintptr_t>(Q) | reinterpret_cast<uintptr_t>(K) |
+                          reinterpret_cast<uintptr_t>(V) | reinterpret_cast<uintptr_t>(Y);
+    if (all & (es - 1)) return OPTIML_ERR_ALIGNMENT;
+    const bool al16 = (all & 15) == 0 && d_model % 8 == 0;
+    const int64_t dk = d_model / heads;
+    const bool fast = mhsa_umma_supported(d_model, heads, (int)dtype, al16);
+    const bool want_fast = h->forced == OPTIML_VARIANT_AUTO ? fast : h->forced != OPTIML_VARIANT_GENERIC;
+    if (want_fast && !fast) return OPTIML_ERR_UNSUPPORTED;
+    if (!want_fast && (dk > kMhsaGenericMaxDk || (int64_t)N * heads > ((int64_t)1 << 32))) return OPTIML_ERR_UNSUPPORTED;
+    DeviceGuard guard(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (h->log)
+        fprintf(stderr, "[optiml] mhsa N=%lld d_model=%lld heads=%lld dtype=%d -> %s\n", (long long)N, (long long)d_model,
+                (long long)heads, (int)dtype, want_fast ? "mhsa_tcgen05" : "mhsa_generic_fma");
+    if (want_fast)
+        return dk == 64 ? launch_mhsa_umma<64>(h, Q, K, V, Y, (int)N, (int)d_model, (int)heads, st)
+                        : launch_mhsa_umma<128>(h, Q, K, V, Y, (int)N, (int)d_model, (int)heads, st);
+    return dtype == OPTIML_F32 ? launch_mhsa_generic<float>(h, Q, K, V, Y, (int)N, (int)d_model, (int)heads, st)
+                               : launch_mhsa_generic<__nv_bfloat16>(h, Q, K, V, Y, (int)N, (int)d_model, (int)heads, st);
 }
 
 optiml_status_t optiml_force_variant(optiml_handle_t h, optiml_variant_t v) {

@@ -213,3 +213,26 @@ def integer_case(M: int, N: int, K: int, dtype: int, act: int, seed: int = 0, am
     B = small_integers(seed, TENSOR_B, K * N, -amax, amax, dtype)
     bias = small_integers(seed, TENSOR_BIAS, N, -amax, amax, dtype)
     return Case(f"int{M}x{N}x{K}", M, N, K, dtype, act, A, B, bias)
+
+
+# ---------------------------------------------------------------- attention inputs
+
+# name -> (N, d_model, heads): the benchmark shapes of the attention row
+MHSA_WORKLOADS = {
+    "a1": (2048, 1024, 16),      # d_k = 64, small enough for the full oracle
+    "a2": (16384, 2048, 16),     # d_k = 128
+    "a3": (16384, 1024, 16),     # d_k = 64
+}
+
+
+def mhsa_inputs(n: int, d_model: int, dtype: int = BF16, seed: int = 0, q_gain: float = 1.0, key_growth: float = 0.0):
+    """Q, K, V of shape (n, d_model) as flat arrays, N(0, 1) entries (tensor ids 10, 11, 12).
+    q_gain scales Q (sharper softmax); key_growth > 0 scales key row j by 1 + key_growth * j / n,
+    so that the largest score of a row tends to arrive late in the sweep over the keys."""
+    def draw(tensor, gain_rows=None, gain=1.0):
+        x = normal(seed, tensor, n * d_model, 1.0, F32).astype(np.float64) * gain
+        if gain_rows is not None:
+            x = (x.reshape(n, d_model) * gain_rows[:, None]).reshape(-1)
+        return x.astype(np.float32) if dtype == F32 else round_to_bf16_bits(x)
+    rows = None if key_growth == 0.0 else 1.0 + key_growth * np.arange(n, dtype=np.float64) / n
+    return draw(10, gain=q_gain), draw(11, gain_rows=rows), draw(12)
