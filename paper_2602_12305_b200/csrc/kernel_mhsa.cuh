@@ -38,26 +38,34 @@ struct MhsaCfg {
     static constexpr int kChunkBytes = 128 * 128;        // 128 rows x 128 bytes
     static constexpr int kTileBytes = kChunks * kChunkBytes;      // one Q tile, K block or V block
     static constexpr int kPBytes = 2 * kChunkBytes;      // 128 x 128 bf16 probabilities
-    static constexpr int kSlots = DK == 64 ? 6 : 3;      // ring slots, each one K or V block
+    // K blocks are released early in an iteration and V blocks late, so each has its own ring:
+    // the next K block has almost a whole iteration to arrive even with a single slot, the V
+    // ring is double-buffered
+    static constexpr int kKSlots = DK == 64 ? 3 : 1;
+    static constexpr int kVSlots = DK == 64 ? 3 : 2;
     static constexpr int kThreads = 320;
     static constexpr int kTmemCols = 512;                // S0, S1: 2 x 128; O0, O1: 2 x DK
     static constexpr int kColS = 0, kColO = 256;
-    static constexpr int kSmemBytes = 256 + 1024 + kQTiles * kTileBytes + kQTiles * kPBytes + kSlots * kTileBytes;
+    static constexpr int kOffP = kQTiles * kTileBytes;
+    static constexpr int kOffK = kOffP + kQTiles * kPBytes;
+    static constexpr int kOffV = kOffK + kKSlots * kTileBytes;
+    static constexpr int kSmemBytes = 256 + 1024 + kOffV + kVSlots * kTileBytes;
     static constexpr float kRescaleThreshold = 8.0f;     // log2 units
 };
 
 struct MhsaShared {
-    uint64_t full[6], empty[6];       // ring slots
+    uint64_t k_full[3], k_empty[3], v_full[3], v_empty[3];
     uint64_t q_full;
-    uint64_t s_full[2], p_full[2], o_final[2];
+    uint64_t s_full[2], s_free[2], p_full[2], pv_done[2];
     uint64_t drain;
     uint32_t tmem_base;
     volatile int abort;
 };
 static_assert(sizeof(MhsaShared) <= 256, "barrier block");
 
-// Wait sites reported on a time-out: 1 producer/free slot, 2 MMA/Q, 3 MMA/K block, 4 MMA/V block,
-// 5 MMA/probabilities, 6 softmax/scores, 7 softmax/final accumulator.
+// Wait sites reported on a time-out: 1 producer/free K slot, 2 producer/free V slot, 3 MMA/Q,
+// 4 MMA/K block, 5 MMA/V block, 6 MMA/scores read, 7 MMA/probabilities, 8 softmax/scores,
+// 9 softmax/previous P V, 10 softmax/final accumulator.
 template <int DK>
 __global__ void __launch_bounds__(MhsaCfg<DK>::kThreads, 1)
 mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -68,9 +76,6 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     MhsaShared* sh = reinterpret_cast<MhsaShared*>(smem_raw);
     const uint32_t data_base = (ptx::smem_u32(smem_raw) + 256 + 1023) & ~1023u;
     uint8_t* data = smem_raw + (data_base - ptx::smem_u32(smem_raw));
-    uint8_t* q_smem = data;                                        // [2][kTileBytes]
-    uint8_t* p_smem = q_smem + C::kQTiles * C::kTileBytes;         // [2][kPBytes]
-    uint8_t* ring = p_smem + C::kQTiles * C::kPBytes;              // [kSlots][kTileBytes]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int head = blockIdx.y;
@@ -78,15 +83,18 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int nblk = (N + C::BKV - 1) / C::BKV;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < C::kSlots; ++s) {
-            ptx::mbar_init(&sh->full[s], 1);
-            ptx::mbar_init(&sh->empty[s], 1);
+        for (int s = 0; s < 3; ++s) {
+            ptx::mbar_init(&sh->k_full[s], 1);
+            ptx::mbar_init(&sh->k_empty[s], 1);
+            ptx::mbar_init(&sh->v_full[s], 1);
+            ptx::mbar_init(&sh->v_empty[s], 1);
         }
         ptx::mbar_init(&sh->q_full, 1);
         for (int t = 0; t < 2; ++t) {
             ptx::mbar_init(&sh->s_full[t], 1);
+            ptx::mbar_init(&sh->s_free[t], C::BQ);
             ptx::mbar_init(&sh->p_full[t], C::BQ);
-            ptx::mbar_init(&sh->o_final[t], 1);
+            ptx::mbar_init(&sh->pv_done[t], 1);
         }
         ptx::mbar_init(&sh->drain, 1);
         sh->abort = 0;
@@ -113,31 +121,41 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             ptx::mbar_arrive_expect_tx(&sh->q_full, C::kQTiles * C::kTileBytes);
             for (int t = 0; t < C::kQTiles; ++t)
                 for (int c = 0; c < C::kChunks; ++c)
-                    ptx::tma_load_2d(q_smem + t * C::kTileBytes + c * C::kChunkBytes, &map_q, &sh->q_full,
+                    ptx::tma_load_2d(data + t * C::kTileBytes + c * C::kChunkBytes, &map_q, &sh->q_full,
                                      head * DK + c * 64, q0 + t * C::BQ);
-            uint32_t it = 0;
             bool ok = true;
-            for (int j = 0; ok && j < nblk; ++j) {
-                for (int kv = 0; kv < 2; ++kv, ++it) {
-                    const int s = it % C::kSlots;
-                    const uint32_t ph = (it / C::kSlots) & 1;
-                    if (sh->abort || !ptx::mbar_wait(&sh->empty[s], ph ^ 1)) { ok = false; break; }
-                    ptx::mbar_arrive_expect_tx(&sh->full[s], C::kTileBytes);
+            int site = 0, j = 0, done_k = 0, done_v = 0;
+            for (; ok && j < nblk; ++j) {
+                {
+                    const int s = j % C::kKSlots;
+                    const uint32_t ph = (j / C::kKSlots) & 1;
+                    if (sh->abort || (site = 1, !ptx::mbar_wait(&sh->k_empty[s], ph ^ 1))) { ok = false; break; }
+                    ptx::mbar_arrive_expect_tx(&sh->k_full[s], C::kTileBytes);
                     for (int c = 0; c < C::kChunks; ++c)
-                        ptx::tma_load_2d(ring + s * C::kTileBytes + c * C::kChunkBytes, kv ? &map_v : &map_k,
-                                         &sh->full[s], head * DK + c * 64, j * C::BKV);
+                        ptx::tma_load_2d(data + C::kOffK + s * C::kTileBytes + c * C::kChunkBytes, &map_k, &sh->k_full[s],
+                                         head * DK + c * 64, j * C::BKV);
+                    done_k = j + 1;
+                }
+                {
+                    const int s = j % C::kVSlots;
+                    const uint32_t ph = (j / C::kVSlots) & 1;
+                    if (sh->abort || (site = 2, !ptx::mbar_wait(&sh->v_empty[s], ph ^ 1))) { ok = false; break; }
+                    ptx::mbar_arrive_expect_tx(&sh->v_full[s], C::kTileBytes);
+                    for (int c = 0; c < C::kChunks; ++c)
+                        ptx::tma_load_2d(data + C::kOffV + s * C::kTileBytes + c * C::kChunkBytes, &map_v, &sh->v_full[s],
+                                         head * DK + c * 64, j * C::BKV);
+                    done_v = j + 1;
                 }
             }
             if (!ok) {
-                report_timeout(status, 1);
+                report_timeout(status, site);
                 sh->abort = 1;
                 // copies already issued must land before the CTA may exit
                 ptx::mbar_wait(&sh->q_full, 0);
-                const uint32_t n_back = it < (uint32_t)C::kSlots ? it : (uint32_t)C::kSlots;
-                for (uint32_t b = 1; b <= n_back; ++b) {
-                    const uint32_t i = it - b;
-                    ptx::mbar_wait(&sh->full[i % C::kSlots], (i / C::kSlots) & 1);
-                }
+                for (int b = 1; b <= C::kKSlots && b <= done_k; ++b)
+                    ptx::mbar_wait(&sh->k_full[(done_k - b) % C::kKSlots], ((done_k - b) / C::kKSlots) & 1);
+                for (int b = 1; b <= C::kVSlots && b <= done_v; ++b)
+                    ptx::mbar_wait(&sh->v_full[(done_v - b) % C::kVSlots], ((done_v - b) / C::kVSlots) & 1);
             }
         }
     } else if (warp == 1) {
@@ -147,13 +165,10 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             constexpr uint32_t idesc_o = ptx::umma_idesc_bf16(C::BQ, DK, false, true);        // P K-major, V MN-major
             bool ok = true;
             int site = 0;
-            auto slot_addr = [&](uint32_t i) { return data_base + (uint32_t)(C::kQTiles * (C::kTileBytes + C::kPBytes)) +
-                                                      (i % C::kSlots) * C::kTileBytes; };
-            auto wait_slot = [&](uint32_t i) { return ptx::mbar_wait(&sh->full[i % C::kSlots], (i / C::kSlots) & 1); };
             // S_t = Q_t K_j^T, contraction over d_k in steps of 16 (32 bytes inside a 128-byte row)
-            auto issue_s = [&](int t, uint32_t k_slot) {
+            auto issue_s = [&](int t, int j) {
                 const uint32_t q_addr = data_base + t * C::kTileBytes;
-                const uint32_t k_addr = slot_addr(k_slot);
+                const uint32_t k_addr = data_base + C::kOffK + (j % C::kKSlots) * C::kTileBytes;
 #pragma unroll
                 for (int ks = 0; ks < DK / 16; ++ks) {
                     const uint32_t off = (ks >> 2) * C::kChunkBytes + (ks & 3) * 32;
@@ -163,41 +178,47 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 ptx::umma_commit(&sh->s_full[t]);
             };
             // O_t (+)= P_t V_j, contraction over the 128 keys in steps of 16 (16 rows of V)
-            auto issue_pv = [&](int t, uint32_t v_slot, bool accumulate) {
-                const uint32_t p_addr = data_base + C::kQTiles * C::kTileBytes + t * C::kPBytes;
-                const uint32_t v_addr = slot_addr(v_slot);
+            auto issue_pv = [&](int t, int j) {
+                const uint32_t p_addr = data_base + C::kOffP + t * C::kPBytes;
+                const uint32_t v_addr = data_base + C::kOffV + (j % C::kVSlots) * C::kTileBytes;
 #pragma unroll
                 for (int ks = 0; ks < C::BKV / 16; ++ks) {
                     const uint32_t p_off = (ks >> 2) * C::kChunkBytes + (ks & 3) * 32;
                     ptx::umma_bf16(tmem_base + C::kColO + t * DK, ptx::umma_smem_desc(p_addr + p_off, 16, 1024),
                                    ptx::umma_smem_desc(v_addr + ks * 2048, C::kChunkBytes, 1024), idesc_o,
-                                   accumulate || ks != 0);
+                                   j != 0 || ks != 0);
                 }
+                ptx::umma_commit(&sh->pv_done[t]);
             };
-            if (sh->abort || (site = 2, !ptx::mbar_wait(&sh->q_full, 0)) || (site = 3, !wait_slot(0))) ok = false;
+            auto k_ready = [&](int j) { return ptx::mbar_wait(&sh->k_full[j % C::kKSlots], (j / C::kKSlots) & 1); };
+            auto v_ready = [&](int j) { return ptx::mbar_wait(&sh->v_full[j % C::kVSlots], (j / C::kVSlots) & 1); };
+            if (sh->abort || (site = 3, !ptx::mbar_wait(&sh->q_full, 0)) || (site = 4, !k_ready(0))) ok = false;
             if (ok) {
                 ptx::tcgen05_fence_after_sync();
                 issue_s(0, 0);
                 issue_s(1, 0);
-                ptx::umma_commit(&sh->empty[0]);
+                ptx::umma_commit(&sh->k_empty[0]);
             }
             for (int j = 0; ok && j < nblk; ++j) {
-                const uint32_t v_it = 2 * j + 1, k_next = 2 * j + 2;
-                for (int t = 0; t < 2; ++t) {
-                    if (sh->abort || (site = 5, !ptx::mbar_wait(&sh->p_full[t], j & 1))) { ok = false; break; }
-                    if (t == 0 && (site = 4, !wait_slot(v_it))) { ok = false; break; }
-                    ptx::tcgen05_fence_after_sync();
-                    issue_pv(t, v_it, j != 0);
-                    if (t == 1) ptx::umma_commit(&sh->empty[v_it % C::kSlots]);
-                    if (j + 1 < nblk) {
-                        if (t == 0 && (site = 3, !wait_slot(k_next))) { ok = false; break; }
+                if (j + 1 < nblk) {
+                    // the scores of block j + 1 as soon as the softmax threads hold block j in registers
+                    if (sh->abort || (site = 4, !k_ready(j + 1))) { ok = false; break; }
+                    for (int t = 0; t < 2; ++t) {
+                        if (sh->abort || (site = 6, !ptx::mbar_wait(&sh->s_free[t], j & 1))) { ok = false; break; }
                         ptx::tcgen05_fence_after_sync();
-                        issue_s(t, k_next);
-                        if (t == 1) ptx::umma_commit(&sh->empty[k_next % C::kSlots]);
-                    } else {
-                        ptx::umma_commit(&sh->o_final[t]);
+                        issue_s(t, j + 1);
                     }
+                    if (!ok) break;
+                    ptx::umma_commit(&sh->k_empty[(j + 1) % C::kKSlots]);
                 }
+                if (sh->abort || (site = 5, !v_ready(j))) { ok = false; break; }
+                for (int t = 0; t < 2; ++t) {
+                    if (sh->abort || (site = 7, !ptx::mbar_wait(&sh->p_full[t], j & 1))) { ok = false; break; }
+                    ptx::tcgen05_fence_after_sync();
+                    issue_pv(t, j);
+                }
+                if (!ok) break;
+                ptx::umma_commit(&sh->v_empty[j % C::kVSlots]);
             }
             if (!ok) {
                 report_timeout(status, site);
@@ -215,74 +236,99 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
         const uint32_t s_addr = lane_base + C::kColS + t * C::BKV;
         const uint32_t o_addr = lane_base + C::kColO + t * DK;
-        uint8_t* p_row = p_smem + t * C::kPBytes + r * 128;
-        float m_used = 0.0f, l = 0.0f;
+        uint8_t* p_row = data + C::kOffP + t * C::kPBytes + r * 128;
+        const float2 scale2 = make_float2(scale_log2, scale_log2);
+        float m_used = 0.0f;
+        float2 l2[2] = {make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f)};
         bool ok = true;
+        int site = 8;
         for (int j = 0; j < nblk; ++j) {
             bool got = !sh->abort && ptx::mbar_wait(&sh->s_full[t], j & 1);
             got = __all_sync(0xffffffffu, got);
             if (!got) { ok = false; break; }
             ptx::tcgen05_fence_after_sync();
-            const int nvalid = min(C::BKV, N - j * C::BKV);
-            // pass 1: row maximum of the valid scores
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                ptx::tmem_ld_32x32(s_addr + c * 32, v);
-                ptx::tmem_ld_wait();
+            // the whole row of scores into registers, then the tensor-memory block is free again
+            uint32_t v[4][32];
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (c * 32 + i < nvalid) mx = fmaxf(mx, __uint_as_float(v[i]));
+            for (int c = 0; c < 4; ++c) ptx::tmem_ld_32x32(s_addr + c * 32, v[c]);
+            ptx::tmem_ld_wait();
+            ptx::tcgen05_fence_before_sync();
+            ptx::mbar_arrive(&sh->s_free[t]);
+            const int nvalid = N - j * C::BKV;
+            if (nvalid < C::BKV) {
+                // keys past the end of the sequence (zero-filled by TMA) take no part
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (c * 32 + i >= nvalid) v[c][i] = __float_as_uint(-INFINITY);
             }
-            mx *= scale_log2;
+            float mx4[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                float a = __uint_as_float(v[c][0]);
+#pragma unroll
+                for (int i = 1; i < 32; i += 2)
+                    a = fmaxf(a, fmaxf(__uint_as_float(v[c][i]), __uint_as_float(v[c][(i + 1) & 31])));
+                mx4[c] = a;
+            }
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
             bool raise = false;
             if (j == 0) {
                 m_used = mx;
             } else if (mx > m_used + C::kRescaleThreshold) {
                 raise = true;
             }
+            bool prev_done = j == 0;                     // has P V of block j - 1 been waited for?
             if (__any_sync(0xffffffffu, raise)) {
-                // every earlier P V of this tile has finished (the MMA that produced these scores
-                // was issued after it), so the accumulator can be rescaled in place
+                // the accumulator is rescaled in place once the previous P V has finished
+                got = !sh->abort && ptx::mbar_wait(&sh->pv_done[t], (j - 1) & 1);
+                got = __all_sync(0xffffffffu, got);
+                if (!got) { ok = false; site = 9; break; }
+                prev_done = true;
+                ptx::tcgen05_fence_after_sync();
                 const float alpha = raise ? ptx::ex2_approx(m_used - mx) : 1.0f;
                 if (raise) {
-                    l *= alpha;
+                    l2[0].x *= alpha; l2[0].y *= alpha; l2[1].x *= alpha; l2[1].y *= alpha;
                     m_used = mx;
                 }
 #pragma unroll 1
                 for (int c = 0; c < DK / 32; ++c) {
-                    uint32_t v[32];
-                    ptx::tmem_ld_32x32(o_addr + c * 32, v);
+                    uint32_t o[32];
+                    ptx::tmem_ld_32x32(o_addr + c * 32, o);
                     ptx::tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-                    ptx::tmem_st_32x32(o_addr + c * 32, v);
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    ptx::tmem_st_32x32(o_addr + c * 32, o);
                 }
                 ptx::tmem_st_wait();
             }
-            // pass 2: probabilities relative to m_used, bf16, into the swizzled K-major P tile
-#pragma unroll 1
+            // probabilities relative to m_used: 2^(s * scale - m), packed to bf16 in place
+            const float2 negm2 = make_float2(-m_used, -m_used);
+#pragma unroll
             for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                ptx::tmem_ld_32x32(s_addr + c * 32, v);
-                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    const float2 x = ptx::ffma2(make_float2(__uint_as_float(v[c][i]), __uint_as_float(v[c][i + 1])), scale2, negm2);
+                    const float2 e = make_float2(ptx::ex2_approx(x.x), ptx::ex2_approx(x.y));
+                    l2[(i >> 1) & 1] = ptx::fadd2(l2[(i >> 1) & 1], e);
+                    v[c][i >> 1] = pack_bf16x2(e.x, e.y);
+                }
+            }
+            if (!prev_done) {
+                // the previous P V still reads this tile's P buffer until it has finished
+                got = !sh->abort && ptx::mbar_wait(&sh->pv_done[t], (j - 1) & 1);
+                got = __all_sync(0xffffffffu, got);
+                if (!got) { ok = false; site = 9; break; }
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
                 uint8_t* atom_row = p_row + (c >> 1) * C::kChunkBytes;
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
-                    uint32_t o[4];
-#pragma unroll
-                    for (int p = 0; p < 4; ++p) {
-                        const int i0 = g * 8 + 2 * p;
-                        float e0 = ptx::ex2_approx(fmaf(__uint_as_float(v[i0]), scale_log2, -m_used));
-                        float e1 = ptx::ex2_approx(fmaf(__uint_as_float(v[i0 + 1]), scale_log2, -m_used));
-                        if (c * 32 + i0 >= nvalid) e0 = 0.0f;
-                        if (c * 32 + i0 + 1 >= nvalid) e1 = 0.0f;
-                        l += e0 + e1;
-                        o[p] = pack_bf16x2(e0, e1);
-                    }
                     const int chunk16 = (c & 1) * 4 + g;
-                    *reinterpret_cast<uint4*>(atom_row + ((chunk16 ^ (lane & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                    *reinterpret_cast<uint4*>(atom_row + ((chunk16 ^ (lane & 7)) << 4)) =
+                        make_uint4(v[c][4 * g], v[c][4 * g + 1], v[c][4 * g + 2], v[c][4 * g + 3]);
                 }
             }
             ptx::fence_proxy_async_smem();
@@ -290,35 +336,33 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             ptx::mbar_arrive(&sh->p_full[t]);
         }
         if (ok) {
-            bool got = !sh->abort && ptx::mbar_wait(&sh->o_final[t], 0);
+            bool got = !sh->abort && ptx::mbar_wait(&sh->pv_done[t], (nblk - 1) & 1);
             got = __all_sync(0xffffffffu, got);
-            if (!got) {
-                ok = false;
-                if (lane == 0) report_timeout(status, 7);
-            }
-        } else if (lane == 0) {
-            report_timeout(status, 6);
+            if (!got) { ok = false; site = 10; }
         }
-        if (!ok) sh->abort = 1;
+        if (!ok) {
+            if (lane == 0) report_timeout(status, site);
+            sh->abort = 1;
+        }
         ptx::griddep_launch_dependents();
         if (ok) {
             ptx::tcgen05_fence_after_sync();
-            const float inv = 1.0f / l;
+            const float inv = 1.0f / ((l2[0].x + l2[0].y) + (l2[1].x + l2[1].y));
             const int row = q0 + t * C::BQ + r;
             __nv_bfloat16* y_row = Y + (size_t)row * d_model + head * DK;
 #pragma unroll 1
             for (int c = 0; c < DK / 32; ++c) {
-                uint32_t v[32];
-                ptx::tmem_ld_32x32(o_addr + c * 32, v);
+                uint32_t o[32];
+                ptx::tmem_ld_32x32(o_addr + c * 32, o);
                 ptx::tmem_ld_wait();
                 if (row < N) {
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
-                        uint32_t o[4];
+                        uint32_t w[4];
 #pragma unroll
                         for (int p = 0; p < 4; ++p)
-                            o[p] = pack_bf16x2(__uint_as_float(v[g * 8 + 2 * p]) * inv, __uint_as_float(v[g * 8 + 2 * p + 1]) * inv);
-                        *reinterpret_cast<uint4*>(y_row + c * 32 + g * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                            w[p] = pack_bf16x2(__uint_as_float(o[g * 8 + 2 * p]) * inv, __uint_as_float(o[g * 8 + 2 * p + 1]) * inv);
+                        *reinterpret_cast<uint4*>(y_row + c * 32 + g * 8) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 }
             }

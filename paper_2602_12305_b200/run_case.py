@@ -4,6 +4,7 @@ profiling (ncu) and for quick timing of a forced variant.
     python -m paper_2602_12305_b200.run_case --workload c3 [--variant auto|0..5] [--iters 3]
         [--M m --N n --K k] [--sets 2] [--time]
     python -m paper_2602_12305_b200.run_case --reduce sum|dot|mse [--n 67108864] [--iters 3]
+    python -m paper_2602_12305_b200.run_case --mhsa a1|a2|a3 [--N n --K d_model --heads h] [--iters 3]
 
 Each iteration uses the next of `--sets` distinct buffer sets.  With --time, CUDA-event
 times per launch are printed (median / min) with the implied TFLOP/s and GB/s.
@@ -49,6 +50,37 @@ def run_reduce(a):
     return 0 if status == binding.OK else 1
 
 
+def run_mhsa(a):
+    n, d_model, heads = synth.MHSA_WORKLOADS[a.mhsa]
+    n, d_model, heads = a.N or n, a.K or d_model, a.heads or heads
+    h = binding.Handle(0)
+    if a.variant != "auto":
+        h.force_variant(int(a.variant))
+    q, k, v = synth.mhsa_inputs(n, d_model, synth.BF16)
+    sets = []
+    for _ in range(a.sets):
+        Q, K, V = (_dev(x, synth.BF16, (n, d_model)) for x in (q, k, v))
+        sets.append((Q, K, V, torch.empty_like(Q)))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(a.warmup):
+        Q, K, V, Y = sets[i % len(sets)]
+        h.mhsa(Q, K, V, heads, Y=Y)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(a.iters):
+        Q, K, V, Y = sets[(a.warmup + i) % len(sets)]
+        h.mhsa(Q, K, V, heads, Y=Y)
+    e1.record()
+    torch.cuda.synchronize()
+    status = h.get_last_status()
+    us = e0.elapsed_time(e1) * 1e3 / a.iters
+    flops = 4 * n * n * d_model
+    print(f"mhsa {a.mhsa} N={n} d_model={d_model} heads={heads}: {a.iters} launches, status {binding.status_string(status)}, "
+          f"{us:.1f} us per launch, {flops / 1e6 / us:.1f} TFLOP/s")
+    h.destroy()
+    return 0 if status == binding.OK else 1
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="c2", choices=sorted(synth.WORKLOADS))
@@ -63,9 +95,13 @@ def main():
     ap.add_argument("--no-step-events", action="store_true", help="one event pair around all launches only")
     ap.add_argument("--reduce", choices=["sum", "dot", "mse"], help="run the stand-alone reduction instead")
     ap.add_argument("--n", type=int, default=1 << 26, help="vector length for --reduce")
+    ap.add_argument("--mhsa", choices=sorted(synth.MHSA_WORKLOADS), help="run multi-head self-attention instead")
+    ap.add_argument("--heads", type=int, help="with --mhsa: override the head count (and --N, --K = d_model)")
     a = ap.parse_args()
     if a.reduce:
         return run_reduce(a)
+    if a.mhsa:
+        return run_mhsa(a)
 
     c = synth.make_case(a.workload, M=a.M, N=a.N, K=a.K)
     h = binding.Handle(0)
