@@ -44,10 +44,14 @@ struct MhsaCfg {
     static constexpr int kKSlots = DK == 64 ? 3 : 1;
     static constexpr int kVSlots = DK == 64 ? 3 : 2;
     static constexpr int kThreads = 320;
-    static constexpr int kTmemCols = 512;                // S0, S1: 2 x 128; O0, O1: 2 x DK
+    static constexpr int kTmemCols = 512;                // S0, S1: 2 x 128; O0, O1: 2 x DK; P0, P1: 2 x 64
     static constexpr int kColS = 0, kColO = 256;
+    // d_k = 64 leaves 128 columns of tensor memory for the probabilities (two bf16 per column),
+    // which the P V product then reads as its A operand; at d_k = 128 they go through shared memory
+    static constexpr bool kPInTmem = DK == 64;
+    static constexpr int kColP = 384;
     static constexpr int kOffP = kQTiles * kTileBytes;
-    static constexpr int kOffK = kOffP + kQTiles * kPBytes;
+    static constexpr int kOffK = kOffP + (kPInTmem ? 0 : kQTiles * kPBytes);
     static constexpr int kOffV = kOffK + kKSlots * kTileBytes;
     static constexpr int kSmemBytes = 256 + 1024 + kOffV + kVSlots * kTileBytes;
     static constexpr float kRescaleThreshold = 8.0f;     // log2 units
@@ -184,9 +188,14 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 #pragma unroll
                 for (int ks = 0; ks < C::BKV / 16; ++ks) {
                     const uint32_t p_off = (ks >> 2) * C::kChunkBytes + (ks & 3) * 32;
-                    ptx::umma_bf16(tmem_base + C::kColO + t * DK, ptx::umma_smem_desc(p_addr + p_off, 16, 1024),
-                                   ptx::umma_smem_desc(v_addr + ks * 2048, C::kChunkBytes, 1024), idesc_o,
-                                   j != 0 || ks != 0);
+                    if (C::kPInTmem)
+                        ptx::umma_bf16_tmem_a(tmem_base + C::kColO + t * DK, tmem_base + C::kColP + t * 64 + ks * 8,
+                                              ptx::umma_smem_desc(v_addr + ks * 2048, C::kChunkBytes, 1024), idesc_o,
+                                              j != 0 || ks != 0);
+                    else
+                        ptx::umma_bf16(tmem_base + C::kColO + t * DK, ptx::umma_smem_desc(p_addr + p_off, 16, 1024),
+                                       ptx::umma_smem_desc(v_addr + ks * 2048, C::kChunkBytes, 1024), idesc_o,
+                                       j != 0 || ks != 0);
                 }
                 ptx::umma_commit(&sh->pv_done[t]);
             };
@@ -321,17 +330,29 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 got = __all_sync(0xffffffffu, got);
                 if (!got) { ok = false; site = 9; break; }
             }
+            if (C::kPInTmem) {
+                // 128 probabilities = 64 packed columns of this thread's lane
+                uint32_t w[32];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint8_t* atom_row = p_row + (c >> 1) * C::kChunkBytes;
+                for (int hh = 0; hh < 2; ++hh) {
 #pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    const int chunk16 = (c & 1) * 4 + g;
-                    *reinterpret_cast<uint4*>(atom_row + ((chunk16 ^ (lane & 7)) << 4)) =
-                        make_uint4(v[c][4 * g], v[c][4 * g + 1], v[c][4 * g + 2], v[c][4 * g + 3]);
+                    for (int i = 0; i < 32; ++i) w[i] = v[2 * hh + (i >> 4)][i & 15];
+                    ptx::tmem_st_32x32(lane_base + C::kColP + t * 64 + hh * 32, w);
                 }
+                ptx::tmem_st_wait();
+            } else {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint8_t* atom_row = p_row + (c >> 1) * C::kChunkBytes;
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        const int chunk16 = (c & 1) * 4 + g;
+                        *reinterpret_cast<uint4*>(atom_row + ((chunk16 ^ (lane & 7)) << 4)) =
+                            make_uint4(v[c][4 * g], v[c][4 * g + 1], v[c][4 * g + 2], v[c][4 * g + 3]);
+                    }
+                }
+                ptx::fence_proxy_async_smem();
             }
-            ptx::fence_proxy_async_smem();
             ptx::tcgen05_fence_before_sync();
             ptx::mbar_arrive(&sh->p_full[t]);
         }
