@@ -48,7 +48,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel,
 # from the ncu captures summarised under profiles/; None = not captured for the current kernel.
 NCU_TRAFFIC_BYTES = {"c1": 542464, "c2": 137573632, "c3": 121340928, "c4": 108860672, "c5": 2799265680,
-                     "sum": 272239616, "dot": 540065280, "mse": None}
+                     "sum": 272239616, "dot": 540065280, "mse": None, "a2": None, "a3": None}
 
 
 def load_peaks():
@@ -429,6 +429,49 @@ def measure_reductions(handle, device, peaks, peak_src, steps, warmup):
     return rows
 
 
+def measure_attention(handle, device, peaks, peak_src, steps, warmup):
+    """Multi-head self-attention (bf16, tensor-core kernel) on the two large synthetic workloads:
+    d_k = 128 and d_k = 64, 16384 rows, 16 heads.  Flops = 4 N^2 d_model (the two products)."""
+    rows = []
+    stream = torch.cuda.current_stream(device)
+    for name in ("a2", "a3"):
+        n, d_model, heads = synth.MHSA_WORKLOADS[name]
+        q, k, v = synth.mhsa_inputs(n, d_model, synth.BF16)
+        nsets = max(2, math.ceil(4 * L2_BYTES / (8 * n * d_model)))
+        sets = []
+        for _ in range(nsets):
+            Q, K, V = (to_device(x, synth.BF16, (n, d_model), device) for x in (q, k, v))
+            sets.append((Q, K, V, torch.empty_like(Q)))
+        k_steps = max(5, min(steps, 100))
+        for i in range(warmup):
+            Q, K, V, Y = sets[i % nsets]
+            handle.mhsa(Q, K, V, heads, Y=Y, stream=stream)
+        torch.cuda.synchronize(device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(k_steps):
+            Q, K, V, Y = sets[(warmup + i) % nsets]
+            handle.mhsa(Q, K, V, heads, Y=Y, stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize(device)
+        from paper_2602_12305_b200 import binding
+        if handle.get_last_status() != binding.OK:
+            raise RuntimeError(f"attention {name}: device-side time-out reported")
+        us = e0.elapsed_time(e1) * 1e3 / k_steps
+        flops = 4.0 * n * n * d_model
+        tf = flops / 1e12 / (us * 1e-6)
+        rows.append({"workload": f"{name}: bf16 self-attention N={n} d_model={d_model} heads={heads} (d_k={d_model // heads})",
+                     "us_per_step": us, "tflops": tf, "steps": k_steps,
+                     "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                  "frac": tf / peaks["bf16_tflops"], "frac_of_sustained": tf / peaks["bf16_tflops_sustained"],
+                                  "traffic": NCU_TRAFFIC_BYTES.get(name), "algorithmic_flops": flops,
+                                  "algorithmic_bytes": 8 * n * d_model,
+                                  "peak_source": f"of {peak_src}: bf16 GEMM burst"}})
+        del sets
+        torch.cuda.empty_cache()
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -489,6 +532,8 @@ def main():
     reductions = [] if args.no_per_shape else measure_reductions(handle, device, peaks, peak_src, min(args.steps, 200),
                                                                  args.warmup)
 
+    attention = [] if args.no_per_shape else measure_attention(handle, device, peaks, peak_src, args.steps, args.warmup)
+
     line = {"metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": region_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32" if case.dtype == synth.F32 else "bf16 inputs, f32 accumulate", "data": "synthetic",
@@ -500,7 +545,7 @@ def main():
                     "d2h_bytes_per_step": main_res["d2h"], "ms_per_step": e2e_ms / main_res["e2e_steps"],
                     "steps": main_res["e2e_steps"]},
             "gpu_launches": main_res["launches"], "replicas": "independent replicas, no data-path collective",
-            "per_shape": per_shape, "reductions": reductions}
+            "per_shape": per_shape, "reductions": reductions, "attention": attention}
     sampler.stop()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(case, unit)

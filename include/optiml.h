@@ -220,6 +220,33 @@ optiml_status_t optiml_force_variant(optiml_handle_t h, optiml_variant_t v);
  * pointers are assumed 16-byte aligned), or -1 on bad arguments. */
 int optiml_select_variant(optiml_handle_t h, int64_t M, int64_t N, int64_t K, optiml_dtype_t dtype);
 
+/*
+ * Tuning options of the streaming kernels (the GEMV-like and skinny shapes, which are bound
+ * by HBM bandwidth, not by arithmetic).  They change how the stream over B is scheduled.  The
+ * prefetch, ring and trigger options never change a result bit; SKINNY_STAGE_ROWS moves the
+ * places where K is cut when a problem is split along K, so partial sums may then round
+ * differently (still one fixed order per setting).  The defaults come from
+ * sweeps on B200; optiml_set_option overrides one for later calls on this handle (values
+ * 0 .. 2^20, else INVALID_ARG), optiml_get_option reads it back (-1 on bad arguments).
+ *
+ * Prefetching "ahead of the dependency wait": kernels are launched as programmatic
+ * dependents, so a kernel's CTAs may start while the previous kernel in the stream still
+ * drains.  They may not read or write anything before that kernel has finished, but they
+ * may ask for lines of B to be brought from DRAM into L2: L2 is where this GPU's own writes
+ * land, so a prefetch that overtakes a writer cannot make a later load see stale data.
+ */
+typedef enum {
+    OPTIML_OPT_GEMV_PREFETCH_ROWS = 0,    /* GEMV: rows of its K slice each CTA prefetches into L2 before the wait */
+    OPTIML_OPT_SKINNY_STAGE_ROWS = 1,     /* skinny: rows of K per pipeline stage, 128 or 192 (192: M <= 32 only)  */
+    OPTIML_OPT_SKINNY_RING_STAGES = 2,    /* skinny: depth of the shared-memory ring of B tiles; 0 = all that fit   */
+    OPTIML_OPT_SKINNY_PREFETCH_EARLY = 3, /* skinny: ring stages of B prefetched into L2 before the wait            */
+    OPTIML_OPT_SKINNY_LATE_TRIGGER = 4,   /* skinny: 1 = release the next kernel's CTAs after a CTA's last load,
+                                             0 = as soon as the kernel starts                                       */
+    OPTIML_OPT_COUNT = 5
+} optiml_option_t;
+optiml_status_t optiml_set_option(optiml_handle_t h, optiml_option_t opt, int64_t value);
+int64_t optiml_get_option(optiml_handle_t h, optiml_option_t opt);
+
 /* Number of kernels launched by this handle since it was created. */
 int64_t optiml_launch_count(optiml_handle_t h);
 

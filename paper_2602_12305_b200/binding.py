@@ -20,6 +20,10 @@ VARIANT_COUNT = 6
 
 REDUCE_SUM, REDUCE_DOT, REDUCE_MSE = 0, 1, 2
 
+(OPT_GEMV_PREFETCH_ROWS, OPT_SKINNY_STAGE_ROWS, OPT_SKINNY_RING_STAGES, OPT_SKINNY_PREFETCH_EARLY,
+ OPT_SKINNY_LATE_TRIGGER) = range(5)
+OPT_COUNT = 5
+
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ARCH, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(8)
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liboptiml_gemm.so")
@@ -38,6 +42,8 @@ EXPORTS = {
     "optiml_force_variant": (_ci, [_vp, _ci]),
     "optiml_select_variant": (_ci, [_vp, _i64, _i64, _i64, _ci]),
     "optiml_launch_count": (_i64, [_vp]),
+    "optiml_set_option": (_ci, [_vp, _ci, _i64]),
+    "optiml_get_option": (_i64, [_vp, _ci]),
     "optiml_status_string": (ctypes.c_char_p, [_ci]),
     "optiml_variant_name": (ctypes.c_char_p, [_ci]),
     "optiml_version": (_ci, []),
@@ -229,3 +235,9 @@ class Handle:
 
     def launch_count(self) -> int:
         return self._lib.optiml_launch_count(self._h)
+
+    def set_option(self, opt: int, value: int):
+        _check(self._lib.optiml_set_option(self._h, int(opt), int(value)), "optiml_set_option")
+
+    def get_option(self, opt: int) -> int:
+        return self._lib.optiml_get_option(self._h, int(opt))

@@ -83,7 +83,8 @@ __device__ __forceinline__ uint4 ld_stream_v4(const void* p) {
 
 // Record a bounded wait that gave up: low byte = status, next byte = which wait (1 producer
 // waiting for a free stage, 2 MMA waiting for a free accumulator, 3 MMA waiting for the A
-// tile, 4 MMA waiting for a filled stage, 5 epilogue waiting for an accumulator), upper
+// tile, 4 MMA waiting for a filled stage, 5 epilogue waiting for an accumulator; 6 is not a wait:
+// the dynamic shared memory of a streaming kernel did not start on a 1024-byte boundary), upper
 // half = CTA index.  The first report wins.
 __device__ __forceinline__ void report_timeout(int* status, int site) {
     atomicCAS(status, kDevOk, kDevTimeout | (site << 8) | ((int)(blockIdx.x & 0x7FFF) << 16));

@@ -47,7 +47,8 @@ __device__ __forceinline__ void gemv_unpack(const uint4& v, float (&b)[4], float
 template <typename T, int MR>
 __global__ void __launch_bounds__(kGemvThreads, gemv_ctas_per_sm(MR))
 gemv_splitk_kernel(const T* __restrict__ A, const T* __restrict__ B, const T* __restrict__ bias, T* __restrict__ Y,
-                   int M, int N, int K, int act, float* __restrict__ partials, unsigned int* __restrict__ counters) {
+                   int M, int N, int K, int act, float* __restrict__ partials, unsigned int* __restrict__ counters,
+                   int prefetch_rows) {
     constexpr int V = GemvVec<T>::V, kCols = GemvVec<T>::kCols;
     __shared__ float red[kGemvWarps][MR][kCols];
     __shared__ int s_last;
@@ -65,7 +66,17 @@ gemv_splitk_kernel(const T* __restrict__ A, const T* __restrict__ B, const T* __
 #pragma unroll
         for (int j = 0; j < V; ++j) acc[m][j] = 0.0f;
 
-    // launched as a programmatic dependent: wait for the previous kernel before touching memory
+    // Launched as a programmatic dependent, this CTA may be running while the previous kernel
+    // still drains.  Nothing may be read or written before the wait below, but the first rows of
+    // this CTA's slice of B can be pulled from DRAM into L2 meanwhile (one 512-byte row segment
+    // per thread and instruction), so that HBM does not idle across the kernel boundary.
+    if (prefetch_rows > 0 && (int64_t)cb * kCols < N) {
+        const int64_t n0 = (int64_t)cb * kCols;
+        const uint32_t seg = (uint32_t)((N - n0 < kCols ? N - n0 : kCols) * (int64_t)sizeof(T));   // multiple of 16
+        const int rows = k_end - k_begin < prefetch_rows ? k_end - k_begin : prefetch_rows;
+        for (int r = threadIdx.x; r < rows; r += kGemvThreads)
+            ptx::prefetch_l2_bulk(B + (int64_t)(k_begin + r) * N + n0, seg);
+    }
     ptx::griddep_wait();
     ptx::griddep_launch_dependents();
 
@@ -129,19 +140,21 @@ gemv_splitk_kernel(const T* __restrict__ A, const T* __restrict__ B, const T* __
         if (!s_last) return;
         __threadfence();
         const float* all = partials + (size_t)cb * S * (MR * kCols);
-        // slices in order, eight loads in flight at a time (one dependent chain of L2 round
-        // trips per slice would cost more than the whole stream over B)
+        // slices in order, kBatch loads in flight at a time (one dependent chain of L2 round
+        // trips per slice would cost more than the whole stream over B; a single row of A leaves
+        // the registers for 24 at once, which covers the 23 slices of 1 x 8192 x 8192 in one trip)
+        constexpr int kBatch = MR == 1 ? 24 : 8;
         if (has_col) {
 #pragma unroll
             for (int m = 0; m < MR; ++m) {
                 float s = 0.0f;
-                for (int q0 = 0; q0 < S; q0 += 8) {
-                    float v[8];
+                for (int q0 = 0; q0 < S; q0 += kBatch) {
+                    float v[kBatch];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
+                    for (int i = 0; i < kBatch; ++i)
                         v[i] = (q0 + i < S) ? __ldcg(all + (size_t)(q0 + i) * (MR * kCols) + m * kCols + t) : 0.0f;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) s += v[i];
+                    for (int i = 0; i < kBatch; ++i) s += v[i];
                 }
                 sum[m] = s;
             }

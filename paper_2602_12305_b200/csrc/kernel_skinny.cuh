@@ -42,40 +42,51 @@
 
 namespace optiml {
 
-template <int MP>
+// MP: padded M (accumulator columns).  SUB: 64-row sub-blocks of K per pipeline stage.
+template <int MP, int SUB>
 struct SkinnyCfg {
     static_assert(MP == 16 || MP == 32 || MP == 64 || MP == 128, "padded M");
+    static_assert(SUB == 2 || SUB == 3, "sub-blocks per stage");
     // One pipeline stage carries kSub sub-blocks of 64 K rows: every stage costs one
     // tcgen05.commit / mbarrier round trip, and with the tiny MMAs of this kernel that round
     // trip, not HBM, limits a 64-row stage.
     // (measured, 16 x 14336 x 4096: 64-row stages 41 us, 128-row 25.7 us, 192-row 23.9 us;
     // larger stages leave too few of them in the ring)
-    static constexpr int kSub = MP <= 32 ? 3 : 2;
+    static constexpr int kSub = SUB;
     static constexpr int BN = 128, BK = 64 * kSub;
     static constexpr int kBChunkBytes = 64 * 64 * 2;           // 64 k-rows x 64 columns: 8 KiB
     static constexpr int kBSubBytes = 2 * kBChunkBytes;        // 64 k-rows x 128 columns
     static constexpr int kBBytes = kSub * kBSubBytes;          // one stage of the B ring
     static constexpr int kASubBytes = MP * 64 * 2;
     static constexpr int kABytes = kSub * kASubBytes;          // one slot of the A ring
-    static constexpr int kFit = (212 * 1024 - kABytes) / (kBBytes + kABytes);
-    static constexpr int kStages = kFit < 12 ? kFit : 12;
-    // The A ring needs no "empty" barrier: a slot is reused kAStages K blocks later, and by
+    static constexpr int kBarrierBytes = 512;                  // SkinnyShared, after the rings
+    static constexpr int kFit = (226 * 1024 - kBarrierBytes - kABytes) / (kBBytes + kABytes);
+    static constexpr int kStages = kFit < 12 ? kFit : 12;      // deepest B ring a CTA can hold
+    // The A ring needs no "empty" barrier: a slot is reused (stages + 1) K blocks later, and by
     // then the producer has waited for B stages whose release implies that every MMA of the
-    // old K block is done (it can be at most kStages stages ahead of the MMAs).
+    // old K block is done (it can be at most `stages` stages ahead of the MMAs).
     static constexpr int kAStages = kStages + 1;
     static constexpr int kThreads = 192;
     static constexpr int kAcc = 256 / MP < 8 ? 256 / MP : 8;   // column tiles per sweep
     static constexpr int kTmemCols = 2 * kAcc * MP;            // 256 (MP = 16) or 512
     static constexpr int kChunk = MP < 32 ? MP : 32;           // accumulator columns per tcgen05.ld
-    static constexpr int kSmemBytes = kStages * kBBytes + kAStages * kABytes + 512 + 1024;
+    // dynamic shared memory of a launch whose B ring is `stages` deep (A ring: one more)
+    static constexpr int smem_bytes(int stages) { return stages * kBBytes + (stages + 1) * kABytes + kBarrierBytes; }
+    static constexpr int kSmemBytes = smem_bytes(kStages);
+    // Deepest ring that lets two CTAs share an SM (228 KiB, 1 KiB reserved per CTA), so that the
+    // next call's CTAs could be resident and set up while this call's CTAs finish; 0 where not
+    // even two stages fit.  (Measured on 16 x 14336 x 4096: such short rings of 128-row stages
+    // lose more, 3-4 us, than the overlap wins; the launcher uses the deepest ring by default.)
+    static constexpr int kFit2 = (113 * 1024 - kBarrierBytes - kABytes) / (kBBytes + kABytes);
+    static constexpr int kStagesShared = kFit2 >= 2 ? kFit2 : 0;
     static constexpr int kSlotFloats = MP * BN;                // one partial tile in scratch
 };
 
-template <int MP>
+template <int MP, int SUB>
 struct SkinnyShared {
-    uint64_t full[SkinnyCfg<MP>::kStages];
-    uint64_t empty[SkinnyCfg<MP>::kStages];
-    uint64_t a_full[SkinnyCfg<MP>::kAStages];
+    uint64_t full[SkinnyCfg<MP, SUB>::kStages];
+    uint64_t empty[SkinnyCfg<MP, SUB>::kStages];
+    uint64_t a_full[SkinnyCfg<MP, SUB>::kAStages];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint64_t drain;
@@ -100,6 +111,40 @@ struct SkinnyPlan {
 
 struct SkinnyRect {
     int t0, t1, kb0, kb1, band;
+};
+
+// Run-time tuning of the streaming pipeline (set per handle; see optiml_set_option).
+struct SkinnyTune {
+    int stages;          // depth of the B ring, 2 .. SkinnyCfg::kStages
+    int prefetch_early;  // units (one stage of B each) prefetched into L2 before the wait on the previous kernel
+    int late_trigger;    // 1: let the next kernel's CTAs start when this CTA has issued its last load
+};
+
+// Walks the units of a CTA's rectangle in the order the pipeline consumes them: chunks of up to
+// kAcc column tiles; within a chunk K-major, the chunk's tiles for every K block.
+template <int kAcc>
+struct SkinnySweep {
+    int tc, kb, j, nt;
+    bool done;
+    __device__ __forceinline__ void start(const SkinnyRect& r) {
+        tc = r.t0;
+        kb = r.kb0;
+        j = 0;
+        nt = min(kAcc, r.t1 - r.t0);
+        done = r.t0 >= r.t1 || r.kb0 >= r.kb1;
+    }
+    __device__ __forceinline__ void next(const SkinnyRect& r) {
+        if (++j < nt) return;
+        j = 0;
+        if (++kb < r.kb1) return;
+        kb = r.kb0;
+        tc += kAcc;
+        if (tc >= r.t1) {
+            done = true;
+            return;
+        }
+        nt = min(kAcc, r.t1 - tc);
+    }
 };
 
 __host__ __device__ __forceinline__ SkinnyRect skinny_rect(const SkinnyPlan& p, int c) {
@@ -221,25 +266,53 @@ inline SkinnyPlan make_skinny_plan(int64_t tiles, int64_t kblocks, int num_sms, 
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-template <int MP>
-__global__ void __launch_bounds__(SkinnyCfg<MP>::kThreads, 1)
+template <int MP, int SUB>
+__global__ void __launch_bounds__(SkinnyCfg<MP, SUB>::kThreads, SkinnyCfg<MP, SUB>::kStagesShared ? 2 : 1)
 gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                         const __nv_bfloat16* __restrict__ bias, __nv_bfloat16* __restrict__ Y, int M, int N, int K,
-                        int act, const __grid_constant__ SkinnyPlan plan, float* __restrict__ partials,
-                        unsigned int* __restrict__ counters, int* __restrict__ status) {
-    using C = SkinnyCfg<MP>;
-    using Sh = SkinnyShared<MP>;
-    static_assert(sizeof(Sh) <= 512, "barrier block");
-    extern __shared__ uint8_t smem_raw[];
-    Sh* sh = reinterpret_cast<Sh*>(smem_raw);
-    const uint32_t ring_base = (ptx::smem_u32(smem_raw) + 512 + 1023) & ~1023u;     // B ring, then A ring
-    uint8_t* ring = smem_raw + (ring_base - ptx::smem_u32(smem_raw));
-    const uint32_t aring_base = ring_base + C::kStages * C::kBBytes;
-    uint8_t* aring = ring + C::kStages * C::kBBytes;
+                        int act, const __grid_constant__ SkinnyPlan plan, const SkinnyTune tune,
+                        float* __restrict__ partials, unsigned int* __restrict__ counters, int* __restrict__ status) {
+    using C = SkinnyCfg<MP, SUB>;
+    using Sh = SkinnyShared<MP, SUB>;
+    static_assert(sizeof(Sh) <= C::kBarrierBytes, "barrier block");
+    // B ring, A ring, barrier block.  The rings hold 128-byte-swizzled tiles and need a 1024-byte
+    // aligned base; no slack is reserved for aligning by hand (it would cost the second CTA per
+    // SM its place), so a base that is not aligned is reported instead of used.
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t ring_base = ptx::smem_u32(smem_raw);
+    if (ring_base & 1023u) {
+        if (threadIdx.x == 0) report_timeout(status, 6);
+        return;
+    }
+    const int kStagesRt = tune.stages, kAStagesRt = tune.stages + 1;   // ring depths of this launch
+    uint8_t* ring = smem_raw;
+    const uint32_t aring_base = ring_base + kStagesRt * C::kBBytes;
+    uint8_t* aring = ring + kStagesRt * C::kBBytes;
+    Sh* sh = reinterpret_cast<Sh*>(aring + kAStagesRt * C::kABytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const SkinnyRect rect = skinny_rect(plan, blockIdx.x);
 
+    // L2 prefetch of B: the first `prefetch_early` units of this CTA's sweep are requested by one
+    // lane BEFORE the wait on the previous kernel.  A prefetch only moves DRAM
+    // lines into L2, so it may overtake that kernel; HBM then stays busy while it drains.
+    // (Prefetching further units ahead of the TMA loads during the sweep was measured too and
+    // only slowed the stream down: the requests pass through the same TMA unit as the loads.)
+    // It comes first of all, and from a warp that has no part in the set-up below, because the
+    // tensor-memory allocation there may have to wait for the previous call's CTA on this SM.
+    if (warp == 2 && lane == 0) {
+        ptx::prefetch_tensormap(&map_a);
+        ptx::prefetch_tensormap(&map_b);
+        SkinnySweep<C::kAcc> pf;
+        pf.start(rect);
+        for (int i = 0; i < tune.prefetch_early && !pf.done; ++i, pf.next(rect)) {
+#pragma unroll
+            for (int u = 0; u < C::kSub; ++u) {
+                ptx::prefetch_l2_tma_2d(&map_b, (pf.tc + pf.j) * C::BN, pf.kb * C::BK + u * 64);
+                ptx::prefetch_l2_tma_2d(&map_b, (pf.tc + pf.j) * C::BN + 64, pf.kb * C::BK + u * 64);
+            }
+        }
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::kStages; ++s) {
             ptx::mbar_init(&sh->full[s], 1);
@@ -262,15 +335,14 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     __syncthreads();
     ptx::tcgen05_fence_after_sync();
     const uint32_t tmem_base = sh->tmem_base;
+
     // set-up above overlapped the previous kernel's tail; from here on global memory is touched
     ptx::griddep_wait();
-    ptx::griddep_launch_dependents();
+    if (!tune.late_trigger) ptx::griddep_launch_dependents();
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            ptx::prefetch_tensormap(&map_a);
-            ptx::prefetch_tensormap(&map_b);
             const uint64_t pol_stream = ptx::policy_evict_first();   // B is read exactly once
             const uint64_t pol_keep = ptx::policy_evict_last();      // A is re-read by every CTA
             uint32_t it = 0, ait = 0;
@@ -279,15 +351,15 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             for (int tc = rect.t0; tc < rect.t1 && ok; tc += C::kAcc) {
                 const int nt = min(C::kAcc, rect.t1 - tc);
                 for (int kb = rect.kb0; kb < rect.kb1 && ok; ++kb, ++ait) {
-                    const int sa = ait % C::kAStages;
+                    const int sa = ait % kAStagesRt;
                     ptx::mbar_arrive_expect_tx(&sh->a_full[sa], C::kABytes);
 #pragma unroll
                     for (int u = 0; u < C::kSub; ++u)
                         ptx::tma_load_2d_hint(aring + sa * C::kABytes + u * C::kASubBytes, &map_a, &sh->a_full[sa],
                                               kb * C::BK + u * 64, 0, pol_keep);
                     for (int j = 0; j < nt; ++j, ++it) {
-                        const int s = it % C::kStages;
-                        if (sh->abort || (site = 1, !ptx::mbar_wait(&sh->empty[s], ((it / C::kStages) & 1) ^ 1))) { ok = false; break; }
+                        const int s = it % kStagesRt;
+                        if (sh->abort || (site = 1, !ptx::mbar_wait(&sh->empty[s], ((it / kStagesRt) & 1) ^ 1))) { ok = false; break; }
                         uint8_t* b_dst = ring + s * C::kBBytes;
                         ptx::mbar_arrive_expect_tx(&sh->full[s], C::kBBytes);
 #pragma unroll
@@ -300,19 +372,22 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                     }
                 }
             }
+            // every load of this CTA is on its way: the next kernel's CTAs may take the SMs that
+            // free up and start their own prefetch while this one computes and stores
+            if (tune.late_trigger) ptx::griddep_launch_dependents();
             if (!ok) {
                 report_timeout(status, site);
                 sh->abort = 1;
                 // copies already issued must land before the CTA may exit
-                const uint32_t n_back = it < (uint32_t)C::kStages ? it : (uint32_t)C::kStages;
+                const uint32_t n_back = it < (uint32_t)kStagesRt ? it : (uint32_t)kStagesRt;
                 for (uint32_t b = 1; b <= n_back; ++b) {
                     const uint32_t j = it - b;
-                    ptx::mbar_wait(&sh->full[j % C::kStages], (j / C::kStages) & 1);
+                    ptx::mbar_wait(&sh->full[j % kStagesRt], (j / kStagesRt) & 1);
                 }
-                const uint32_t a_back = ait < (uint32_t)C::kAStages ? ait : (uint32_t)C::kAStages;
+                const uint32_t a_back = ait < (uint32_t)kAStagesRt ? ait : (uint32_t)kAStagesRt;
                 for (uint32_t b = 1; b <= a_back; ++b) {
                     const uint32_t j = ait - b;
-                    ptx::mbar_wait(&sh->a_full[j % C::kAStages], (j / C::kAStages) & 1);
+                    ptx::mbar_wait(&sh->a_full[j % kAStagesRt], (j / kAStagesRt) & 1);
                 }
             }
         }
@@ -329,12 +404,12 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 if (sh->abort || (site = 2, !ptx::mbar_wait(&sh->tmem_empty[half], ((chunk_it >> 1) & 1) ^ 1))) { ok = false; break; }
                 ptx::tcgen05_fence_after_sync();
                 for (int kb = rect.kb0; kb < rect.kb1 && ok; ++kb, ++ait) {
-                    const int sa = ait % C::kAStages;
-                    if (sh->abort || (site = 3, !ptx::mbar_wait(&sh->a_full[sa], (ait / C::kAStages) & 1))) { ok = false; break; }
+                    const int sa = ait % kAStagesRt;
+                    if (sh->abort || (site = 3, !ptx::mbar_wait(&sh->a_full[sa], (ait / kAStagesRt) & 1))) { ok = false; break; }
                     const uint32_t a_addr = aring_base + sa * C::kABytes;            // tile of A
                     for (int j = 0; j < nt; ++j, ++it) {
-                        const int s = it % C::kStages;
-                        if (sh->abort || (site = 4, !ptx::mbar_wait(&sh->full[s], (it / C::kStages) & 1))) { ok = false; break; }
+                        const int s = it % kStagesRt;
+                        if (sh->abort || (site = 4, !ptx::mbar_wait(&sh->full[s], (it / kStagesRt) & 1))) { ok = false; break; }
                         ptx::tcgen05_fence_after_sync();
                         const uint32_t b_addr = ring_base + s * C::kBBytes;          // tile of B
                         const uint32_t d_tmem = tmem_base + (half * C::kAcc + j) * MP;

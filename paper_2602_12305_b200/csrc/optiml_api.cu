@@ -32,6 +32,17 @@ constexpr int kVersion = 10000 * 0 + 100 * 1 + 0;
 constexpr size_t kPartialBytes = (size_t)32 << 20;   // split-K / stream-K partial sums
 constexpr int kNumCounters = 1 << 16;                 // one arrival counter per column block / tile
 constexpr int kMapCache = 32;
+// Defaults of the tuning options (optiml_option_t order), chosen from sweeps on B200.
+constexpr int64_t kOptionDefaults[OPTIML_OPT_COUNT] = {
+    // 1 x 8192 x 8192 bf16: 22.8 us without prefetch, 21.7-21.9 us with 48-96 rows, 23.9 us with 192
+    /* GEMV_PREFETCH_ROWS    */ 96,
+    // 16 x 14336 x 4096: 128-row stages 26.8-27.1 us at any ring depth, 192-row stages 23.5 us;
+    // two stages prefetched before the wait and the late trigger: 22.9 us
+    /* SKINNY_STAGE_ROWS     */ 192,
+    /* SKINNY_RING_STAGES    */ 0,
+    /* SKINNY_PREFETCH_EARLY */ 2,
+    /* SKINNY_LATE_TRIGGER   */ 1,
+};
 
 typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                     const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -72,6 +83,7 @@ struct optiml_handle_s {
     int next_map = 0;
     void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
     size_t stage_bytes[4] = {0, 0, 0, 0};
+    int64_t options[OPTIML_OPT_COUNT];
 };
 
 namespace {
@@ -227,16 +239,17 @@ optiml_status_t launch_f32(optiml_handle_t h, const void* A, const void* B, cons
 
 template <int MR>
 void launch_gemv_mr(const void* A, const void* B, const void* bias, void* Y, int M, int N, int K, int act, dim3 grid,
-                    float* partials, unsigned int* counters, cudaStream_t st) {
+                    float* partials, unsigned int* counters, int prefetch_rows, cudaStream_t st) {
     launch_pdl(gemv_splitk_kernel<__nv_bfloat16, MR>, grid, dim3(kGemvThreads), 0, st, (const __nv_bfloat16*)A,
-               (const __nv_bfloat16*)B, (const __nv_bfloat16*)bias, (__nv_bfloat16*)Y, M, N, K, act, partials, counters);
+               (const __nv_bfloat16*)B, (const __nv_bfloat16*)bias, (__nv_bfloat16*)Y, M, N, K, act, partials, counters,
+               prefetch_rows);
 }
 
 template <int MR>
 void launch_gemv_f32_mr(const void* A, const void* B, const void* bias, void* Y, int M, int N, int K, int act, dim3 grid,
-                        float* partials, unsigned int* counters, cudaStream_t st) {
+                        float* partials, unsigned int* counters, int prefetch_rows, cudaStream_t st) {
     launch_pdl(gemv_splitk_kernel<float, MR>, grid, dim3(kGemvThreads), 0, st, (const float*)A, (const float*)B,
-               (const float*)bias, (float*)Y, M, N, K, act, partials, counters);
+               (const float*)bias, (float*)Y, M, N, K, act, partials, counters, prefetch_rows);
 }
 
 optiml_status_t launch_gemv(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
@@ -253,23 +266,24 @@ optiml_status_t launch_gemv(optiml_handle_t h, const void* A, const void* B, con
     if (S > 65535) S = 65535;
     if (S < 1) S = 1;
     dim3 grid((unsigned)col_blocks, (unsigned)S);
+    const int pf = (int)h->options[OPTIML_OPT_GEMV_PREFETCH_ROWS];
     if (dtype == OPTIML_F32) {
-        if (MR == 1) launch_gemv_f32_mr<1>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
-        else if (MR == 2) launch_gemv_f32_mr<2>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
-        else launch_gemv_f32_mr<4>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
+        if (MR == 1) launch_gemv_f32_mr<1>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, pf, st);
+        else if (MR == 2) launch_gemv_f32_mr<2>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, pf, st);
+        else launch_gemv_f32_mr<4>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, pf, st);
     } else {
-        if (MR == 1) launch_gemv_mr<1>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
-        else if (MR == 2) launch_gemv_mr<2>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
-        else launch_gemv_mr<4>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, st);
+        if (MR == 1) launch_gemv_mr<1>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, pf, st);
+        else if (MR == 2) launch_gemv_mr<2>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, pf, st);
+        else launch_gemv_mr<4>(A, B, bias, Y, M, N, K, act, grid, h->partials, h->counters, pf, st);
     }
     h->launches += 1;
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
 }
 
-template <int MP>
-optiml_status_t launch_skinny_mp(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M,
-                                 int N, int K, int act, cudaStream_t st) {
-    using C = SkinnyCfg<MP>;
+template <int MP, int SUB>
+optiml_status_t launch_skinny_cfg(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M,
+                                  int N, int K, int act, cudaStream_t st) {
+    using C = SkinnyCfg<MP, SUB>;
     const CUtensorMap* ma = get_map(h, A, (uint64_t)M, (uint64_t)K, MP, 64);
     const CUtensorMap* mb = get_map(h, B, (uint64_t)K, (uint64_t)N, 64, 64);
     if (!ma || !mb) return OPTIML_ERR_CUDA;
@@ -277,10 +291,27 @@ optiml_status_t launch_skinny_mp(optiml_handle_t h, const void* A, const void* B
     // one unit = one K block of one column tile; a CTA streams it at about 58 GB/s
     const double unit_us = (double)(C::kBBytes + C::kABytes) / 58.0e3;
     const SkinnyPlan plan = make_skinny_plan(ceil_div64(N, C::BN), ceil_div64(K, C::BK), h->num_sms, max_slots, unit_us);
-    launch_pdl(gemm_skinny_umma_kernel<MP>, dim3(plan.G), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb,
-               (const __nv_bfloat16*)bias, (__nv_bfloat16*)Y, M, N, K, act, plan, h->partials, h->counters, h->status);
+    SkinnyTune tune;
+    const int64_t want = h->options[OPTIML_OPT_SKINNY_RING_STAGES];
+    tune.stages = want < 2 || want > C::kStages ? C::kStages : (int)want;
+    tune.prefetch_early = (int)h->options[OPTIML_OPT_SKINNY_PREFETCH_EARLY];
+    tune.late_trigger = h->options[OPTIML_OPT_SKINNY_LATE_TRIGGER] != 0;
+    launch_pdl(gemm_skinny_umma_kernel<MP, SUB>, dim3(plan.G), dim3(C::kThreads), C::smem_bytes(tune.stages), st, *ma,
+               *mb, (const __nv_bfloat16*)bias, (__nv_bfloat16*)Y, M, N, K, act, plan, tune, h->partials, h->counters,
+               h->status);
     h->launches += 1;
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+// Rows of K per pipeline stage: 128 or 192 (option SKINNY_STAGE_ROWS; 192 only up to 32 rows of A).
+template <int MP>
+optiml_status_t launch_skinny_mp(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M,
+                                 int N, int K, int act, cudaStream_t st) {
+    if constexpr (MP <= 32) {
+        if (h->options[OPTIML_OPT_SKINNY_STAGE_ROWS] == 192)
+            return launch_skinny_cfg<MP, 3>(h, A, B, bias, Y, M, N, K, act, st);
+    }
+    return launch_skinny_cfg<MP, 2>(h, A, B, bias, Y, M, N, K, act, st);
 }
 
 optiml_status_t launch_skinny(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
@@ -363,6 +394,15 @@ bool set_smem(F* fn, int bytes) {
     return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
 }
 
+// Streaming kernels: the whole shared-memory carve-out (with a short ring, option
+// SKINNY_RING_STAGES, this call's and the next call's CTAs can then share an SM).
+template <typename F>
+bool set_skinny(F* fn, int bytes) {
+    return set_smem(fn, bytes) &&
+           cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) ==
+               cudaSuccess;
+}
+
 bool configure_kernels() {
     bool ok = true;
     ok &= set_smem(gemm_umma_kernel<kActNone>, UmmaCfg::kSmemBytes);
@@ -373,10 +413,12 @@ bool configure_kernels() {
     ok &= set_smem(gemm_umma2_kernel<kActRelu>, Umma2Cfg::kSmemBytes);
     ok &= set_smem(gemm_umma2_kernel<kActGeluTanh>, Umma2Cfg::kSmemBytes);
     ok &= set_smem(gemm_umma2_kernel<kActSigmoid>, Umma2Cfg::kSmemBytes);
-    ok &= set_smem(gemm_skinny_umma_kernel<16>, SkinnyCfg<16>::kSmemBytes);
-    ok &= set_smem(gemm_skinny_umma_kernel<32>, SkinnyCfg<32>::kSmemBytes);
-    ok &= set_smem(gemm_skinny_umma_kernel<64>, SkinnyCfg<64>::kSmemBytes);
-    ok &= set_smem(gemm_skinny_umma_kernel<128>, SkinnyCfg<128>::kSmemBytes);
+    ok &= set_skinny(gemm_skinny_umma_kernel<16, 2>, SkinnyCfg<16, 2>::kSmemBytes);
+    ok &= set_skinny(gemm_skinny_umma_kernel<16, 3>, SkinnyCfg<16, 3>::kSmemBytes);
+    ok &= set_skinny(gemm_skinny_umma_kernel<32, 2>, SkinnyCfg<32, 2>::kSmemBytes);
+    ok &= set_skinny(gemm_skinny_umma_kernel<32, 3>, SkinnyCfg<32, 3>::kSmemBytes);
+    ok &= set_skinny(gemm_skinny_umma_kernel<64, 2>, SkinnyCfg<64, 2>::kSmemBytes);
+    ok &= set_skinny(gemm_skinny_umma_kernel<128, 2>, SkinnyCfg<128, 2>::kSmemBytes);
     ok &= set_smem(mhsa_umma_kernel<64>, MhsaCfg<64>::kSmemBytes);
     ok &= set_smem(mhsa_umma_kernel<128>, MhsaCfg<128>::kSmemBytes);
     return ok;
@@ -446,6 +488,7 @@ optiml_status_t optiml_create(optiml_handle_t* out, int device) {
     h->num_sms = prop.multiProcessorCount;
     const char* lg = getenv("OPTIML_LOG");
     h->log = lg && lg[0] == '1';
+    for (int i = 0; i < OPTIML_OPT_COUNT; ++i) h->options[i] = kOptionDefaults[i];
 
     DeviceGuard guard(device);
     cudaDriverEntryPointQueryResult qres;
@@ -650,6 +693,18 @@ int optiml_select_variant(optiml_handle_t h, int64_t M, int64_t N, int64_t K, op
 
 int64_t optiml_launch_count(optiml_handle_t h) { return h ? h->launches : -1; }
 
+optiml_status_t optiml_set_option(optiml_handle_t h, optiml_option_t opt, int64_t value) {
+    if (!h || (int)opt < 0 || (int)opt >= OPTIML_OPT_COUNT) return OPTIML_ERR_INVALID_ARG;
+    if (value < 0 || value > (1 << 20)) return OPTIML_ERR_INVALID_ARG;
+    h->options[opt] = value;
+    return OPTIML_OK;
+}
+
+int64_t optiml_get_option(optiml_handle_t h, optiml_option_t opt) {
+    if (!h || (int)opt < 0 || (int)opt >= OPTIML_OPT_COUNT) return -1;
+    return h->options[opt];
+}
+
 const char* optiml_status_string(optiml_status_t s) {
     switch (s) {
     case OPTIML_OK: return "ok";
@@ -747,9 +802,9 @@ optiml_status_t optiml_gemv_noalloc(const void* A, const void* B, const void* bi
     // (the partial sums need not: every slot that is read is written first).
     if (cudaMemsetAsync(counters, 0, kNoAllocCounterBytes, st) != cudaSuccess) return OPTIML_ERR_CUDA;
     dim3 grid((unsigned)col_blocks, (unsigned)S);
-    if (MR == 1) launch_gemv_mr<1>(A, B, bias, Y, m, n, k, (int)act, grid, partials, counters, st);
-    else if (MR == 2) launch_gemv_mr<2>(A, B, bias, Y, m, n, k, (int)act, grid, partials, counters, st);
-    else launch_gemv_mr<4>(A, B, bias, Y, m, n, k, (int)act, grid, partials, counters, st);
+    if (MR == 1) launch_gemv_mr<1>(A, B, bias, Y, m, n, k, (int)act, grid, partials, counters, 0, st);
+    else if (MR == 2) launch_gemv_mr<2>(A, B, bias, Y, m, n, k, (int)act, grid, partials, counters, 0, st);
+    else launch_gemv_mr<4>(A, B, bias, Y, m, n, k, (int)act, grid, partials, counters, 0, st);
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
 }
 

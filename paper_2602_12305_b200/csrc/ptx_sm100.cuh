@@ -80,6 +80,24 @@ __device__ __forceinline__ void griddep_launch_dependents() {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// ---------------------------------------------------------------- L2 prefetch
+//
+// Prefetches move data from DRAM into L2 and nothing else: no register, no shared memory, no
+// completion to wait for.  L2 is the point of coherence for this GPU's own writes, so a
+// prefetch may be issued BEFORE griddep_wait(): if the previous kernel has yet to write the
+// line, its later write lands in the same L2 line and the load after the wait sees it.
+// The streaming kernels use this to keep HBM busy while the previous kernel drains.
+
+// `bytes` contiguous bytes at `p`; both multiples of 16.
+__device__ __forceinline__ void prefetch_l2_bulk(const void* p, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+// One box of a tiled tensor map (same coordinates and alignment rule as tma_load_2d).
+__device__ __forceinline__ void prefetch_l2_tma_2d(const CUtensorMap* map, int x, int y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y)
+                 : "memory");
+}
+
 // ---------------------------------------------------------------- proxies / fences
 
 // Make generic-proxy writes to shared memory visible to the async proxy (TMA, tcgen05).

@@ -61,6 +61,8 @@ def test_null_arguments_are_rejected_before_any_cuda_call(lib):
     assert lib.optiml_force_variant(None, 0) == binding.ERR_INVALID_ARG
     assert lib.optiml_select_variant(None, 1, 1, 1, 0) == -1
     assert lib.optiml_launch_count(None) == -1
+    assert lib.optiml_set_option(None, 0, 1) == binding.ERR_INVALID_ARG
+    assert lib.optiml_get_option(None, 0) == -1
 
 
 @pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU behaviour")

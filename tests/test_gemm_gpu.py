@@ -313,3 +313,41 @@ def test_many_shapes_back_to_back_leave_the_scratch_clean(handle):
         for c, r in zip(cases, refs):
             _, y = H.run_case(handle, c)
             H.check_tolerance(y, r, c.dtype, "interleaved")
+
+
+# ---------------------------------------------------------------- tuning options of the streaming kernels
+
+def test_option_arguments(handle):
+    for opt in range(V.OPT_COUNT):
+        assert handle.get_option(opt) >= 0
+    with pytest.raises(binding.OptimlError):
+        handle.set_option(V.OPT_COUNT, 1)
+    with pytest.raises(binding.OptimlError):
+        handle.set_option(V.OPT_GEMV_PREFETCH_ROWS, -1)
+    assert handle.get_option(V.OPT_COUNT) == -1
+
+
+@pytest.mark.parametrize("name,M,N,K,variant", [("c2", 1, 2056, 3000, V.VARIANT_GEMV_SPLITK),
+                                                 ("c2", 3, 520, 777, V.VARIANT_GEMV_SPLITK),
+                                                 ("c3", 16, 1160, 1096, V.VARIANT_SKINNY_UMMA),
+                                                 ("c3", 40, 2312, 4104, V.VARIANT_SKINNY_UMMA)])
+def test_scheduling_options_leave_the_bits_alone(handle, name, M, N, K, variant):
+    """Prefetch depth, ring depth and trigger point only reschedule the stream over B: every
+    setting must match the oracle and give the very same bits; the stage height may move the
+    K cuts of a split problem, so it is held to the tolerance only."""
+    case = synth.make_case(name, M=M, N=N, K=K)
+    saved = [handle.get_option(o) for o in range(V.OPT_COUNT)]
+    try:
+        ref_bits = {}
+        for rows in (128, 192):
+            for pf_rows, stages, early, late in ((0, 0, 0, 0), (1, 2, 1, 1), (64, 3, 5, 0), (100000, 9, 1000, 1)):
+                handle.set_option(V.OPT_GEMV_PREFETCH_ROWS, pf_rows)
+                handle.set_option(V.OPT_SKINNY_STAGE_ROWS, rows)
+                handle.set_option(V.OPT_SKINNY_RING_STAGES, stages)
+                handle.set_option(V.OPT_SKINNY_PREFETCH_EARLY, early)
+                handle.set_option(V.OPT_SKINNY_LATE_TRIGGER, late)
+                bits = parity(handle, case, variant, what=f"{name} {M}x{N}x{K} options {(rows, pf_rows, stages, early, late)}")
+                assert np.array_equal(ref_bits.setdefault(rows, bits), bits)
+    finally:
+        for o, v in enumerate(saved):
+            handle.set_option(o, v)
