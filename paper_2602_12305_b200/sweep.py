@@ -6,6 +6,13 @@ evidence behind the dispatcher's thresholds.
 Prints one markdown table row per M: microseconds per launch of each variant (mean over
 `--iters` back-to-back launches between two CUDA events, rotating over buffer sets larger
 than L2 together) and the variant the dispatcher picks.
+
+    python -m paper_2602_12305_b200.sweep --options [--iters 1000]
+
+Times the two streaming workloads (c2: 1 x 8192 x 8192, c3: 16 x 14336 x 4096) over a grid of
+the tuning options of optiml_set_option (L2 prefetch ahead of the dependency wait, stage height,
+ring depth, trigger point): the evidence behind their defaults.  Also checks that the scheduling
+options leave the output bits alone.
 """
 from __future__ import annotations
 
@@ -50,13 +57,59 @@ def time_variant(h, variant, sets, M, N, K, act, iters):
     return e0.elapsed_time(e1) * 1e3 / iters
 
 
+def sweep_options(iters):
+    h = binding.Handle(0)
+    opts = [binding.OPT_GEMV_PREFETCH_ROWS, binding.OPT_SKINNY_STAGE_ROWS, binding.OPT_SKINNY_RING_STAGES,
+            binding.OPT_SKINNY_PREFETCH_EARLY, binding.OPT_SKINNY_LATE_TRIGGER]
+    defaults = [h.get_option(o) for o in opts]
+
+    def make_sets(c):
+        n = max(2, math.ceil(4 * 126 * 2**20 / c.algorithmic_bytes))
+        A0, B0, b0 = _dev(c.A, (c.M, c.K)), _dev(c.B, (c.K, c.N)), _dev(c.bias, (c.N,))
+        return [(A0.clone(), B0.clone(), b0.clone(), torch.empty((c.M, c.N), dtype=torch.bfloat16, device="cuda"))
+                for _ in range(n)]
+
+    def run(c, sets, variant, values):
+        for o, v in zip(opts, values):
+            h.set_option(o, v)
+        t = min(time_variant(h, variant, sets, c.M, c.N, c.K, c.act, iters) for _ in range(2))
+        return t, sets[0][3].clone()
+
+    print(f"defaults: gemv_prefetch_rows={defaults[0]} stage_rows={defaults[1]} ring_stages={defaults[2]} "
+          f"prefetch_early={defaults[3]} late_trigger={defaults[4]}; best of two runs of {iters} back-to-back launches\n")
+    c = synth.make_case("c2")
+    sets = make_sets(c)
+    print("c2: bf16 1 x 8192 x 8192, GEMV kernel\n\n| rows prefetched before the wait | us per launch | GB/s | same bits |\n|---|---|---|---|")
+    ref = None
+    for rows in (0, 16, 32, 48, 64, 96, 128, 192, 256):
+        t, y = run(c, sets, binding.VARIANT_GEMV_SPLITK, [rows] + defaults[1:])
+        ref = y if ref is None else ref
+        print(f"| {rows} | {t:.2f} | {c.algorithmic_bytes / t / 1e3:.0f} | {bool(torch.equal(ref, y))} |", flush=True)
+    del sets
+    torch.cuda.empty_cache()
+    c = synth.make_case("c3")
+    sets = make_sets(c)
+    print("\nc3: bf16 16 x 14336 x 4096, skinny kernel\n\n| stage rows | ring stages | stages prefetched before the wait | late trigger | us per launch | GB/s | same bits |\n|---|---|---|---|---|---|---|")
+    ref = {}
+    for rows, stage_list in ((192, (2, 3, 4)), (128, (2, 3, 6))):
+        for stages in stage_list:
+            for early, late in ((0, 0), (0, 1), (2, 0), (2, 1), (4, 1), (8, 1)):
+                t, y = run(c, sets, binding.VARIANT_SKINNY_UMMA, [defaults[0], rows, stages, early, late])
+                same = bool(torch.equal(ref.setdefault(rows, y), y))
+                print(f"| {rows} | {stages} | {early} | {late} | {t:.2f} | {c.algorithmic_bytes / t / 1e3:.0f} | {same} |", flush=True)
+    h.destroy()
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--options", action="store_true", help="sweep the streaming kernels' tuning options instead")
     ap.add_argument("--N", type=int, default=8192)
     ap.add_argument("--K", type=int, default=8192)
     ap.add_argument("--Ms", default="1,2,4,8,16,32,64,96,128,192,256,512,1024")
     ap.add_argument("--iters", type=int, default=100)
     a = ap.parse_args()
+    if a.options:
+        return sweep_options(max(a.iters, 1000))
     h = binding.Handle(0)
     act = synth.ACT_RELU
     print(f"N = {a.N}, K = {a.K}, bf16, bias + ReLU; microseconds per launch\n")
