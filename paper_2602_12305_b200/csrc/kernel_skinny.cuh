@@ -66,9 +66,16 @@ struct SkinnyCfg {
     // then the producer has waited for B stages whose release implies that every MMA of the
     // old K block is done (it can be at most `stages` stages ahead of the MMAs).
     static constexpr int kAStages = kStages + 1;
-    static constexpr int kThreads = 192;
+    // MMA-issuing lanes.  A tcgen05.mma with so small an N costs its issuer about 60 cycles, the
+    // tensor pipe under 40, and the issuer also waits on the barriers of every stage: measured
+    // on 16 x 14336 x 4096, one lane needed 0.9 us per 192-row stage, which capped a CTA at
+    // 53 GB/s.  With two lanes each issues every other 16-row step of K into an accumulator of
+    // its own (the epilogue adds the two, always in the same order).  Tensor memory has room for
+    // the second set of accumulators only at MP = 16.
+    static constexpr int kIssuers = MP == 16 ? 2 : 1;
+    static constexpr int kThreads = 192 + 32 * (kIssuers - 1); // warp 6: the second issuing lane
     static constexpr int kAcc = 256 / MP < 8 ? 256 / MP : 8;   // column tiles per sweep
-    static constexpr int kTmemCols = 2 * kAcc * MP;            // 256 (MP = 16) or 512
+    static constexpr int kTmemCols = 2 * kAcc * MP * kIssuers; // 512 in every configuration
     static constexpr int kChunk = MP < 32 ? MP : 32;           // accumulator columns per tcgen05.ld
     // dynamic shared memory of a launch whose B ring is `stages` deep (A ring: one more)
     static constexpr int smem_bytes(int stages) { return stages * kBBytes + (stages + 1) * kABytes + kBarrierBytes; }
@@ -266,6 +273,14 @@ inline SkinnyPlan make_skinny_plan(int64_t tiles, int64_t kblocks, int num_sms, 
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
+// First tensor-memory column of the accumulator of issuing lane w, accumulator set `half`
+// (alternating between sweeps), column tile j of the sweep.
+template <int MP, int SUB>
+__device__ __forceinline__ uint32_t skinny_acc_col(int w, int half, int j) {
+    using C = SkinnyCfg<MP, SUB>;
+    return (uint32_t)(((w * 2 + half) * C::kAcc + j) * MP);
+}
+
 template <int MP, int SUB>
 __global__ void __launch_bounds__(SkinnyCfg<MP, SUB>::kThreads, SkinnyCfg<MP, SUB>::kStagesShared ? 2 : 1)
 gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -316,14 +331,14 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::kStages; ++s) {
             ptx::mbar_init(&sh->full[s], 1);
-            ptx::mbar_init(&sh->empty[s], 1);
+            ptx::mbar_init(&sh->empty[s], C::kIssuers);       // one commit per issuing lane
         }
         for (int s = 0; s < C::kAStages; ++s) ptx::mbar_init(&sh->a_full[s], 1);
         for (int a = 0; a < 2; ++a) {
-            ptx::mbar_init(&sh->tmem_full[a], 1);
+            ptx::mbar_init(&sh->tmem_full[a], C::kIssuers);
             ptx::mbar_init(&sh->tmem_empty[a], 128);
         }
-        ptx::mbar_init(&sh->drain, 1);
+        ptx::mbar_init(&sh->drain, C::kIssuers);
         sh->abort = 0;
         ptx::fence_mbar_init();
     }
@@ -391,10 +406,12 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
+    } else if (warp == 1 || warp == 6) {
+        // ------------------------------------------------------------ MMA issuers
+        // (warp 6 exists only where C::kIssuers == 2)
         if (lane == 0) {
             constexpr uint32_t idesc = ptx::umma_idesc_bf16(C::BN, MP, /*a_mn_major=*/true, /*b_mn_major=*/false);
+            const int w = warp == 1 ? 0 : 1;                  // this lane takes the K steps w, w + kIssuers, ...
             uint32_t it = 0, ait = 0, chunk_it = 0;
             bool ok = true;
             int site = 0;
@@ -412,14 +429,15 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                         if (sh->abort || (site = 4, !ptx::mbar_wait(&sh->full[s], (it / kStagesRt) & 1))) { ok = false; break; }
                         ptx::tcgen05_fence_after_sync();
                         const uint32_t b_addr = ring_base + s * C::kBBytes;          // tile of B
-                        const uint32_t d_tmem = tmem_base + (half * C::kAcc + j) * MP;
+                        const uint32_t d_tmem = tmem_base + skinny_acc_col<MP, SUB>(w, half, j);
 #pragma unroll
-                        for (int k4 = 0; k4 < C::BK / 16; ++k4) {
+                        for (int q = 0; q < C::BK / 16 / C::kIssuers; ++q) {
+                            const int k4 = q * C::kIssuers + w;
                             const uint64_t da = ptx::umma_smem_desc(b_addr + (k4 / 4) * C::kBSubBytes + (k4 % 4) * 2048,
                                                                     C::kBChunkBytes, 1024);
                             const uint64_t db = ptx::umma_smem_desc(a_addr + (k4 / 4) * C::kASubBytes + (k4 % 4) * 32,
                                                                     16, 1024);
-                            ptx::umma_bf16(d_tmem, da, db, idesc, (kb != rect.kb0) || (k4 != 0));
+                            ptx::umma_bf16(d_tmem, da, db, idesc, (kb != rect.kb0) || (q != 0));
                         }
                         ptx::umma_commit(&sh->empty[s]);
                     }
@@ -464,10 +482,19 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
 #pragma unroll 1
                 for (int m0 = 0; m0 < MP; m0 += C::kChunk) {
                     uint32_t v[C::kChunk];
-                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (half * C::kAcc + j) * MP + m0;
+                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + skinny_acc_col<MP, SUB>(0, half, j) + m0;
                     if constexpr (C::kChunk == 16) ptx::tmem_ld_32x16(taddr, v);
                     else ptx::tmem_ld_32x32(taddr, v);
-                    ptx::tmem_ld_wait();
+                    if constexpr (C::kIssuers == 2) {
+                        // the second lane's share of K: acc0 + acc1, always in this order
+                        uint32_t v1[C::kChunk];
+                        ptx::tmem_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + skinny_acc_col<MP, SUB>(1, half, j) + m0, v1);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < C::kChunk; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + __uint_as_float(v1[i]));
+                    } else {
+                        ptx::tmem_ld_wait();
+                    }
                     if (whole) {
 #pragma unroll
                         for (int i = 0; i < C::kChunk; ++i) {
