@@ -238,7 +238,7 @@ int optiml_select_variant(optiml_handle_t h, int64_t M, int64_t N, int64_t K, op
 typedef enum {
     OPTIML_OPT_GEMV_PREFETCH_ROWS = 0,    /* GEMV: rows of its K slice each CTA prefetches into L2 before the wait */
     OPTIML_OPT_SKINNY_STAGE_ROWS = 1,     /* skinny: rows of K per pipeline stage, 128 or 192 (192: M <= 32 only)  */
-    OPTIML_OPT_SKINNY_RING_STAGES = 2,    /* skinny: depth of the shared-memory ring of B tiles; 0 = all that fit   */
+    OPTIML_OPT_SKINNY_RING_STAGES = 2,    /* skinny: depth of the shared-memory ring of B tiles; 0 = the tuned depth */
     OPTIML_OPT_SKINNY_PREFETCH_EARLY = 3, /* skinny: ring stages of B prefetched into L2 before the wait            */
     OPTIML_OPT_SKINNY_LATE_TRIGGER = 4,   /* skinny: 1 = release the next kernel's CTAs after a CTA's last load,
                                              0 = as soon as the kernel starts                                       */

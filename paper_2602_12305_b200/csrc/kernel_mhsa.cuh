@@ -8,9 +8,13 @@
 // accumulator stays in tensor memory for the whole sweep over the keys (online softmax with a
 // running maximum).  Warp roles:
 //   warp 0      TMA producer: the two 128-row Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring
-//   warp 1      one lane issues every MMA: S_t,j = Q_t K_j^T and O_t += P_t,j V_j for t = 0, 1
+//   warp 1      one lane issues the MMAs of query tile 0: S_0,j = Q_0 K_j^T and O_0 += P_0,j V_j
 //   warps 2-5   softmax + output for query tile 0 (one thread per query row = one TMEM lane)
 //   warps 6-9   the same for query tile 1
+//   warp 10     one lane issues the MMAs of query tile 1
+// (One lane for both tiles was the bottleneck: a tcgen05.mma costs its issuer about 60 cycles and
+// every block also costs it six barrier waits, about 3000 cycles per key block in all, more than
+// the tensor pipe or the special-function unit need.)
 // The two query tiles alternate on the tensor pipe: while one tile's threads exponentiate, the
 // other tile's MMAs run.  The running maximum is only raised when a row's new maximum exceeds it
 // by more than 2^8 (in the exp2 domain): the accumulator is then rescaled in tensor memory;
@@ -43,7 +47,7 @@ struct MhsaCfg {
     // ring is double-buffered
     static constexpr int kKSlots = DK == 64 ? 3 : 1;
     static constexpr int kVSlots = DK == 64 ? 3 : 2;
-    static constexpr int kThreads = 320;
+    static constexpr int kThreads = 352;                 // 11 warps: producer, MMA lane of tile 0, 8 softmax warps, MMA lane of tile 1
     static constexpr int kTmemCols = 512;                // S0, S1: 2 x 128; O0, O1: 2 x DK; P0, P1: 2 x 64
     static constexpr int kColS = 0, kColO = 256;
     // d_k = 64 leaves 128 columns of tensor memory for the probabilities (two bf16 per column),
@@ -89,9 +93,9 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     if (threadIdx.x == 0) {
         for (int s = 0; s < 3; ++s) {
             ptx::mbar_init(&sh->k_full[s], 1);
-            ptx::mbar_init(&sh->k_empty[s], 1);
+            ptx::mbar_init(&sh->k_empty[s], 2);            // released by both tiles' MMA lanes
             ptx::mbar_init(&sh->v_full[s], 1);
-            ptx::mbar_init(&sh->v_empty[s], 1);
+            ptx::mbar_init(&sh->v_empty[s], 2);
         }
         ptx::mbar_init(&sh->q_full, 1);
         for (int t = 0; t < 2; ++t) {
@@ -100,7 +104,7 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             ptx::mbar_init(&sh->p_full[t], C::BQ);
             ptx::mbar_init(&sh->pv_done[t], 1);
         }
-        ptx::mbar_init(&sh->drain, 1);
+        ptx::mbar_init(&sh->drain, 2);
         sh->abort = 0;
         ptx::fence_mbar_init();
     }
@@ -162,9 +166,10 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     ptx::mbar_wait(&sh->v_full[(done_v - b) % C::kVSlots], ((done_v - b) / C::kVSlots) & 1);
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
+    } else if (warp == 1 || warp == 10) {
+        // ------------------------------------------------------------ MMA issuers, one per query tile
         if (lane == 0) {
+            const int t = warp == 1 ? 0 : 1;
             constexpr uint32_t idesc_s = ptx::umma_idesc_bf16(C::BQ, C::BKV, false, false);   // Q, K: both K-major
             constexpr uint32_t idesc_o = ptx::umma_idesc_bf16(C::BQ, DK, false, true);        // P K-major, V MN-major
             bool ok = true;
@@ -204,29 +209,22 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             if (sh->abort || (site = 3, !ptx::mbar_wait(&sh->q_full, 0)) || (site = 4, !k_ready(0))) ok = false;
             if (ok) {
                 ptx::tcgen05_fence_after_sync();
-                issue_s(0, 0);
-                issue_s(1, 0);
+                issue_s(t, 0);
                 ptx::umma_commit(&sh->k_empty[0]);
             }
             for (int j = 0; ok && j < nblk; ++j) {
                 if (j + 1 < nblk) {
                     // the scores of block j + 1 as soon as the softmax threads hold block j in registers
                     if (sh->abort || (site = 4, !k_ready(j + 1))) { ok = false; break; }
-                    for (int t = 0; t < 2; ++t) {
-                        if (sh->abort || (site = 6, !ptx::mbar_wait(&sh->s_free[t], j & 1))) { ok = false; break; }
-                        ptx::tcgen05_fence_after_sync();
-                        issue_s(t, j + 1);
-                    }
-                    if (!ok) break;
+                    if (sh->abort || (site = 6, !ptx::mbar_wait(&sh->s_free[t], j & 1))) { ok = false; break; }
+                    ptx::tcgen05_fence_after_sync();
+                    issue_s(t, j + 1);
                     ptx::umma_commit(&sh->k_empty[(j + 1) % C::kKSlots]);
                 }
                 if (sh->abort || (site = 5, !v_ready(j))) { ok = false; break; }
-                for (int t = 0; t < 2; ++t) {
-                    if (sh->abort || (site = 7, !ptx::mbar_wait(&sh->p_full[t], j & 1))) { ok = false; break; }
-                    ptx::tcgen05_fence_after_sync();
-                    issue_pv(t, j);
-                }
-                if (!ok) break;
+                if (sh->abort || (site = 7, !ptx::mbar_wait(&sh->p_full[t], j & 1))) { ok = false; break; }
+                ptx::tcgen05_fence_after_sync();
+                issue_pv(t, j);
                 ptx::umma_commit(&sh->v_empty[j % C::kVSlots]);
             }
             if (!ok) {

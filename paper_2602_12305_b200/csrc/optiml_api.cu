@@ -36,11 +36,11 @@ constexpr int kMapCache = 32;
 constexpr int64_t kOptionDefaults[OPTIML_OPT_COUNT] = {
     // 1 x 8192 x 8192 bf16: 22.8 us without prefetch, 21.7-21.9 us with 48-96 rows, 23.9 us with 192
     /* GEMV_PREFETCH_ROWS    */ 96,
-    // 16 x 14336 x 4096: 128-row stages 26.8-27.1 us at any ring depth, 192-row stages 23.5 us;
-    // two stages prefetched before the wait and the late trigger: 22.9 us
+    // 16 x 14336 x 4096 (two MMA lanes): 128-row stages 22.0-22.4 us, 192-row stages 20.9 us;
+    // four stages prefetched before the wait and the late trigger: 19.9 us
     /* SKINNY_STAGE_ROWS     */ 192,
     /* SKINNY_RING_STAGES    */ 0,
-    /* SKINNY_PREFETCH_EARLY */ 2,
+    /* SKINNY_PREFETCH_EARLY */ 4,
     /* SKINNY_LATE_TRIGGER   */ 1,
 };
 
@@ -293,7 +293,10 @@ optiml_status_t launch_skinny_cfg(optiml_handle_t h, const void* A, const void* 
     const SkinnyPlan plan = make_skinny_plan(ceil_div64(N, C::BN), ceil_div64(K, C::BK), h->num_sms, max_slots, unit_us);
     SkinnyTune tune;
     const int64_t want = h->options[OPTIML_OPT_SKINNY_RING_STAGES];
-    tune.stages = want < 2 || want > C::kStages ? C::kStages : (int)want;
+    // default depth: all that fit, except three 192-row stages at M <= 16 (measured on 16 x 14336 x 4096
+    // with two MMA lanes: 2 / 3 / 4 stages 21.6 / 19.9 / 20.2 us)
+    const int dflt = (MP == 16 && SUB == 3 && C::kStages > 3) ? 3 : C::kStages;
+    tune.stages = want < 2 ? dflt : (want > C::kStages ? C::kStages : (int)want);
     tune.prefetch_early = (int)h->options[OPTIML_OPT_SKINNY_PREFETCH_EARLY];
     tune.late_trigger = h->options[OPTIML_OPT_SKINNY_LATE_TRIGGER] != 0;
     launch_pdl(gemm_skinny_umma_kernel<MP, SUB>, dim3(plan.G), dim3(C::kThreads), C::smem_bytes(tune.stages), st, *ma,
