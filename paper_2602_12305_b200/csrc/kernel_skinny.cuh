@@ -70,11 +70,13 @@ struct SkinnyCfg {
     // tensor pipe under 40, and the issuer also waits on the barriers of every stage: measured
     // on 16 x 14336 x 4096, one lane needed 0.9 us per 192-row stage, which capped a CTA at
     // 53 GB/s.  With two lanes each issues every other 16-row step of K into an accumulator of
-    // its own (the epilogue adds the two, always in the same order).  Tensor memory has room for
-    // the second set of accumulators only at MP = 16.
-    static constexpr int kIssuers = MP == 16 ? 2 : 1;
+    // its own (the epilogue adds the two, always in the same order).  The second set of
+    // accumulators halves the column tiles a sweep can hold (kAcc); at MP = 128 the MMAs are
+    // long enough (N = 128: 64 cycles on the pipe) for one lane.
+    static constexpr int kIssuers = MP <= 64 ? 2 : 1;
     static constexpr int kThreads = 192 + 32 * (kIssuers - 1); // warp 6: the second issuing lane
-    static constexpr int kAcc = 256 / MP < 8 ? 256 / MP : 8;   // column tiles per sweep
+    static constexpr int kAccFit = 256 / (MP * kIssuers);
+    static constexpr int kAcc = kAccFit < 8 ? kAccFit : 8;     // column tiles per sweep
     static constexpr int kTmemCols = 2 * kAcc * MP * kIssuers; // 512 in every configuration
     static constexpr int kChunk = MP < 32 ? MP : 32;           // accumulator columns per tcgen05.ld
     // dynamic shared memory of a launch whose B ring is `stages` deep (A ring: one more)
@@ -488,7 +490,9 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                     if constexpr (C::kIssuers == 2) {
                         // the second lane's share of K: acc0 + acc1, always in this order
                         uint32_t v1[C::kChunk];
-                        ptx::tmem_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + skinny_acc_col<MP, SUB>(1, half, j) + m0, v1);
+                        const uint32_t taddr1 = tmem_base + ((uint32_t)(q * 32) << 16) + skinny_acc_col<MP, SUB>(1, half, j) + m0;
+                        if constexpr (C::kChunk == 16) ptx::tmem_ld_32x16(taddr1, v1);
+                        else ptx::tmem_ld_32x32(taddr1, v1);
                         ptx::tmem_ld_wait();
 #pragma unroll
                         for (int i = 0; i < C::kChunk; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + __uint_as_float(v1[i]));
