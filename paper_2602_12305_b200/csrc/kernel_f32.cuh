@@ -10,6 +10,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "ptx_sm100.cuh"
 
 namespace optiml {
 
@@ -43,6 +44,24 @@ gemm_f32_tiled_kernel(const float* __restrict__ A, const float* __restrict__ B, 
     const int tiles_n = (N + BN - 1) / BN;
     const int64_t m0 = (int64_t)(blockIdx.x / tiles_n) * BM;
     const int64_t n0 = (int64_t)(blockIdx.x % tiles_n) * BN;
+
+    // Launched as a programmatic dependent: before the wait on the previous kernel nothing may be
+    // read, but this CTA's rows of A and columns of B can be pulled into L2 (a prefetch cannot
+    // make a later load stale), so that the dependent global-load round trips of the K loop below
+    // are L2 hits instead of DRAM accesses.  Small problems are pure latency: this is most of it.
+    if (KS > 1) {
+        for (int r = tid; r < BM; r += C::kThreads) {                 // A: BM rows of K floats
+            const int64_t m = m0 + r;
+            if (m < M) {
+                const float* row = A + m * K;
+                for (int64_t k = 0; k < K; k += 4096) ptx::prefetch_l2_bulk(row + k, (uint32_t)((K - k < 4096 ? K - k : 4096) * 4));
+            }
+        }
+        const uint32_t seg = (uint32_t)((N - n0 < BN ? N - n0 : BN) * 4);     // B: K rows of BN floats
+        for (int k = tid; k < K; k += C::kThreads) ptx::prefetch_l2_bulk(B + (int64_t)k * N + n0, seg);
+    }
+    ptx::griddep_wait();
+    ptx::griddep_launch_dependents();
 
     // K is cut into KS contiguous slices of whole BK steps.
     const int steps_total = (K + kF32BK - 1) / kF32BK;

@@ -208,16 +208,16 @@ optiml_status_t launch_f32_cfg(optiml_handle_t h, const float* A, const float* B
     const size_t smem = C::kSmemFloats * sizeof(float);
     switch (act) {
     case OPTIML_ACT_RELU:
-        gemm_f32_tiled_kernel<BM, BN, TM, TN, KS, kActRelu><<<(unsigned)tiles, C::kThreads, smem, st>>>(A, B, bias, Y, M, N, K);
+        launch_pdl(gemm_f32_tiled_kernel<BM, BN, TM, TN, KS, kActRelu>, dim3((unsigned)tiles), dim3(C::kThreads), smem, st, A, B, bias, Y, M, N, K);
         break;
     case OPTIML_ACT_GELU_TANH:
-        gemm_f32_tiled_kernel<BM, BN, TM, TN, KS, kActGeluTanh><<<(unsigned)tiles, C::kThreads, smem, st>>>(A, B, bias, Y, M, N, K);
+        launch_pdl(gemm_f32_tiled_kernel<BM, BN, TM, TN, KS, kActGeluTanh>, dim3((unsigned)tiles), dim3(C::kThreads), smem, st, A, B, bias, Y, M, N, K);
         break;
     case OPTIML_ACT_SIGMOID:
-        gemm_f32_tiled_kernel<BM, BN, TM, TN, KS, kActSigmoid><<<(unsigned)tiles, C::kThreads, smem, st>>>(A, B, bias, Y, M, N, K);
+        launch_pdl(gemm_f32_tiled_kernel<BM, BN, TM, TN, KS, kActSigmoid>, dim3((unsigned)tiles), dim3(C::kThreads), smem, st, A, B, bias, Y, M, N, K);
         break;
     default:
-        gemm_f32_tiled_kernel<BM, BN, TM, TN, KS, kActNone><<<(unsigned)tiles, C::kThreads, smem, st>>>(A, B, bias, Y, M, N, K);
+        launch_pdl(gemm_f32_tiled_kernel<BM, BN, TM, TN, KS, kActNone>, dim3((unsigned)tiles), dim3(C::kThreads), smem, st, A, B, bias, Y, M, N, K);
         break;
     }
     h->launches += 1;
@@ -234,6 +234,7 @@ optiml_status_t launch_f32(optiml_handle_t h, const void* A, const void* B, cons
         return launch_f32_cfg<128, 128, 8, 8, 1>(h, a, b, bi, y, M, N, K, act, st);
     if (ceil_div64(M, 64) * ceil_div64(N, 64) >= h->num_sms)
         return launch_f32_cfg<64, 64, 4, 4, 1>(h, a, b, bi, y, M, N, K, act, st);
+    // (8 or 16 slices of K per CTA instead of 4 were measured too: 5.6 and 6.2 us against 5.4 us on 256^3)
     return launch_f32_cfg<32, 32, 4, 4, 4>(h, a, b, bi, y, M, N, K, act, st);
 }
 
