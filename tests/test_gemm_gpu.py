@@ -351,3 +351,56 @@ def test_scheduling_options_leave_the_bits_alone(handle, name, M, N, K, variant)
     finally:
         for o, v in enumerate(saved):
             handle.set_option(o, v)
+
+
+# ---------------------------------------------------------------- stream order across the dependency wait
+
+@pytest.mark.parametrize("name,M,N,K,variant", [("c2", 1, 2056, 3000, V.VARIANT_GEMV_SPLITK),
+                                                 ("c3", 16, 1160, 1096, V.VARIANT_SKINNY_UMMA),
+                                                 ("c1", 64, 96, 256, V.VARIANT_F32_TILED),
+                                                 ("c4", 300, 520, 264, V.VARIANT_UMMA_2CTA)])
+def test_operands_written_just_before_the_call_are_seen(handle, name, M, N, K, variant):
+    """The streaming kernels ask L2 for lines of B before they wait for the previous kernel in the
+    stream.  That must never show stale data: B (and A, bias) are overwritten on the same stream
+    immediately before each call, alternating between two contents, with no synchronisation in
+    between, and every output must be the one of the contents written last."""
+    cases = [synth.make_case(name, M=M, N=N, K=K, seed=s) for s in (0, 1)]
+    refs = [H.oracle_full(c) for c in cases]
+    dt = cases[0].dtype
+    src = [(H.to_device(c.A, dt, (M, K)), H.to_device(c.B, dt, (K, N)), H.to_device(c.bias, dt, (N,))) for c in cases]
+    A, B, bias = (torch.empty_like(x) for x in src[0])
+    handle.force_variant(variant)
+    outs = []
+    for i in range(12):
+        a, b, bb = src[i & 1]
+        A.copy_(a)
+        B.copy_(b)
+        bias.copy_(bb)
+        outs.append((i & 1, handle.gemm_epilogue(A, B, bias, cases[0].act)))
+    torch.cuda.synchronize()
+    assert handle.get_last_status() == binding.OK
+    for which, Y in outs:
+        y = oracle.widen(H.to_host_bits(Y, dt), dt)
+        H.check_tolerance(y, refs[which], dt, f"{name} {M}x{N}x{K}, contents {which}")
+
+
+def test_chained_calls_consume_the_previous_output(handle):
+    """Y1 = act(A B1) feeds the next call as its A operand with nothing in between: the second
+    kernel is resident while the first still runs and must wait for its output."""
+    M, K1, N1, N2 = 16, 1096, 1160, 1288
+    c1 = synth.make_case("c3", M=M, N=N1, K=K1, act=GELU)
+    c2 = synth.make_case("c3", M=M, N=N2, K=N1, seed=3)
+    A, B1, b1 = H.to_device(c1.A, BF16, (M, K1)), H.to_device(c1.B, BF16, (K1, N1)), H.to_device(c1.bias, BF16, (N1,))
+    B2, b2 = H.to_device(c2.B, BF16, (N1, N2)), H.to_device(c2.bias, BF16, (N2,))
+    results = []
+    for _ in range(6):
+        Y1 = handle.gemm_epilogue(A, B1, b1, GELU)
+        Y2 = handle.gemm_epilogue(Y1, B2, b2, RELU)
+        results.append((Y1, Y2))
+    torch.cuda.synchronize()
+    assert handle.get_last_status() == binding.OK
+    for Y1, Y2 in results:
+        y1_bits = H.to_host_bits(Y1, BF16)
+        H.check_tolerance(oracle.widen(y1_bits, BF16), H.oracle_full(c1), BF16, "first call")
+        ref2 = oracle.gemm_epilogue(y1_bits.reshape(-1), c2.B, c2.bias, M, N2, N1, BF16, RELU)
+        H.check_tolerance(oracle.widen(H.to_host_bits(Y2, BF16), BF16), ref2, BF16, "second call on the first call's output")
