@@ -166,26 +166,27 @@ gemm_umma2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         if (lane == 0) {
             ptx::prefetch_tensormap(&map_a);
             ptx::prefetch_tensormap(&map_b);
-            uint32_t it = 0;
+            uint32_t it = 0, s = 0, ph = 0;
             bool ok = true;
             int site = 0;
             UmmaWork w;
+            // the leader's "full" barriers as seen from this CTA (consecutive 8-byte words)
+            const uint32_t full_leader0 = ptx::mapa_shared(ptx::smem_u32(&sh->full[0]), 0);
             for (int wi = 0; ok && umma2_work_item(plan, pair, wi, w); ++wi) {
                 const int tm = w.tm, tn = w.tn;
+                if (sh->abort) { ok = false; break; }
                 for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
-                    const int s = it % C::kStages;
-                    const uint32_t ph = (it / C::kStages) & 1;
-                    if (sh->abort || (site = 1, !ptx::mbar_wait(&sh->empty[s], ph ^ 1))) { ok = false; break; }
+                    if ((site = 1, !ptx::mbar_wait(&sh->empty[s], ph ^ 1))) { ok = false; break; }
                     uint8_t* a_dst = ring + s * C::kStageBytes;
                     uint8_t* b_dst = a_dst + C::kABytes;
-                    // the leader's "full" barrier of this stage, as seen from this CTA
-                    const uint32_t full_leader = ptx::mapa_shared(ptx::smem_u32(&sh->full[s]), 0);
+                    const uint32_t full_leader = full_leader0 + 8u * s;
                     ptx::mbar_arrive_expect_tx_cluster(full_leader, C::kStageBytes);
                     ptx::tma_load_2d_2cta(a_dst, &map_a, full_leader, kb * C::BK, tm * C::BM + (int)rank * 128);
 #pragma unroll
                     for (int j = 0; j < 2; ++j)
                         ptx::tma_load_2d_2cta(b_dst + j * C::kBChunkBytes, &map_b, full_leader,
                                               tn * C::BN + (int)rank * 128 + j * 64, kb * C::BK);
+                    if (++s == C::kStages) { s = 0; ph ^= 1; }
                 }
             }
             if (!ok) {
@@ -207,7 +208,16 @@ gemm_umma2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0 && rank == 0) {
             constexpr uint32_t idesc = ptx::umma_idesc_bf16(C::BM, C::BN, /*a_mn_major=*/false, /*b_mn_major=*/true);
-            uint32_t it = 0, tile_it = 0;
+            // The issuing lane is on the critical path (a K block costs it the barrier wait plus four
+            // MMA issues, against 512 cycles on the tensor pipe), so its loop is kept lean: the low
+            // words of the shared-memory descriptors advance by constants from stage to stage and
+            // from K step to K step (start address in 16-byte units: A 2 per 16 k, B 128 per 16 k), the
+            // high word never changes, and the stage index wraps by comparison instead of a division.
+            constexpr uint32_t kDescHi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);   // stride 1024 B, version 1, 128-B swizzle
+            const uint32_t a_lo0 = ((ring_base & 0x3FFFFu) >> 4) | ((16u >> 4) << 16);
+            const uint32_t b_lo0 = (((ring_base + C::kABytes) & 0x3FFFFu) >> 4) | ((uint32_t)(C::kBChunkBytes >> 4) << 16);
+            auto desc = [](uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; };
+            uint32_t it = 0, tile_it = 0, s = 0, ph = 0;
             bool ok = true;
             int site = 0;
             UmmaWork w;
@@ -218,23 +228,21 @@ gemm_umma2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 ptx::tcgen05_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + a * C::BN;
                 for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
-                    const int s = it % C::kStages;
-                    const uint32_t ph = (it / C::kStages) & 1;
-                    if (sh->abort || (site = 4, !ptx::mbar_wait(&sh->full[s], ph))) { ok = false; break; }
+                    // (the abort flag is looked at once per tile, above: every wait is bounded anyway)
+                    if ((site = 4, !ptx::mbar_wait(&sh->full[s], ph))) { ok = false; break; }
                     ptx::tcgen05_fence_after_sync();
-                    const uint32_t a_addr = ring_base + s * C::kStageBytes;
-                    const uint32_t b_addr = a_addr + C::kABytes;
+                    const uint32_t a_lo = a_lo0 + s * (uint32_t)(C::kStageBytes >> 4);
+                    const uint32_t b_lo = b_lo0 + s * (uint32_t)(C::kStageBytes >> 4);
+                    // Each descriptor names this CTA's half; the peer's half sits at the same
+                    // shared-memory offsets in the peer CTA.
+                    // A: K-major, 16 k = 32 bytes along the 128-byte row.
+                    // B: MN-major, 16 k = 16 rows of 128 bytes; 64-column chunks 8 KiB apart.
+                    ptx::umma_bf16_2cta(d_tmem, desc(a_lo), desc(b_lo), idesc, kb != w.kb0);
 #pragma unroll
-                    for (int k4 = 0; k4 < C::BK / 16; ++k4) {
-                        // Each descriptor names this CTA's half; the peer's half sits at the same
-                        // shared-memory offsets in the peer CTA.
-                        // A: K-major, 16 k = 32 bytes along the 128-byte row.
-                        // B: MN-major, 16 k = 16 rows of 128 bytes; 64-column chunks 8 KiB apart.
-                        const uint64_t a_desc = ptx::umma_smem_desc(a_addr + k4 * 32, 16, 1024);
-                        const uint64_t b_desc = ptx::umma_smem_desc(b_addr + k4 * 2048, C::kBChunkBytes, 1024);
-                        ptx::umma_bf16_2cta(d_tmem, a_desc, b_desc, idesc, (kb != w.kb0) || (k4 != 0));
-                    }
+                    for (int k4 = 1; k4 < C::BK / 16; ++k4)
+                        ptx::umma_bf16_2cta_acc(d_tmem, desc(a_lo + 2 * k4), desc(b_lo + 128 * k4), idesc);
                     ptx::umma_commit_2cta(&sh->empty[s]);    // both CTAs: stage reusable once these MMAs have read it
+                    if (++s == C::kStages) { s = 0; ph ^= 1; }
                 }
                 if (ok) ptx::umma_commit_2cta(&sh->tmem_full[a]);
             }

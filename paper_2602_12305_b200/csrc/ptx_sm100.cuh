@@ -352,6 +352,11 @@ __device__ __forceinline__ void umma_bf16_2cta(uint32_t d_tmem, uint64_t a_desc,
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// The same, always accumulating onto D (no predicate to set up: one instruction less on the issuing lane).
+__device__ __forceinline__ void umma_bf16_2cta_acc(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+    asm volatile("tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, 1;" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc)
+                 : "memory");
+}
 // Arrive on the barrier at this shared-memory offset in BOTH CTAs of the pair once every
 // tcgen05.mma issued so far has finished.
 __device__ __forceinline__ void umma_commit_2cta(uint64_t* bar) {
