@@ -33,10 +33,19 @@
 namespace optiml {
 
 struct Umma2Cfg {
-    static constexpr int BM = 256, BN = 256, BK = 64, kStages = 6;   // tile of the CTA pair
-    static constexpr int kABytes = 128 * BK * 2;             // this CTA's 128 rows of A: 16 KiB
-    static constexpr int kBChunkBytes = BK * 64 * 2;         // one 64-column chunk: 8 KiB
-    static constexpr int kBBytes = 2 * kBChunkBytes;         // this CTA's 128 columns of B: 16 KiB
+#ifndef OPTIML_UMMA2_SUBK
+#define OPTIML_UMMA2_SUBK 1
+#endif
+    // A stage holds kSubK sub-blocks of 64 k.  Every stage costs each issuing lane one barrier
+    // round trip, but three 128-k stages measured no better than six 64-k stages (4096^3: 103.4
+    // against 101.6 us; 8192 x 8192 x 16384: 1505 against 1491 us), so the finer ring stays.
+    static constexpr int kSubK = OPTIML_UMMA2_SUBK;
+    static constexpr int BM = 256, BN = 256, BK = 64 * kSubK, kStages = 6 / kSubK;   // tile of the CTA pair
+    static constexpr int kASubBytes = 128 * 64 * 2;          // this CTA's 128 rows x 64 k of A: 16 KiB
+    static constexpr int kABytes = kSubK * kASubBytes;
+    static constexpr int kBChunkBytes = 64 * 64 * 2;         // 64 k x one 64-column chunk: 8 KiB
+    static constexpr int kBSubBytes = 2 * kBChunkBytes;      // 64 k x this CTA's 128 columns of B: 16 KiB
+    static constexpr int kBBytes = kSubK * kBSubBytes;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kThreads = 192;
     static constexpr int kTmemCols = 512;
@@ -58,7 +67,8 @@ inline UmmaPlan make_umma2_plan(int64_t M, int64_t N, int64_t K, int num_sms) {
     if (r > 0) {
         split = (int)(pairs / r);
         if (split > 8) split = 8;
-        if (split > p.num_kb / 4) split = p.num_kb / 4;
+        if (split > p.num_kb * Umma2Cfg::kSubK / 4) split = p.num_kb * Umma2Cfg::kSubK / 4;   // at least 256 k per slice
+        if (split > p.num_kb) split = p.num_kb;
         if (split < 1) split = 1;
     }
     if (split == 1) {
@@ -181,11 +191,15 @@ gemm_umma2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     uint8_t* b_dst = a_dst + C::kABytes;
                     const uint32_t full_leader = full_leader0 + 8u * s;
                     ptx::mbar_arrive_expect_tx_cluster(full_leader, C::kStageBytes);
-                    ptx::tma_load_2d_2cta(a_dst, &map_a, full_leader, kb * C::BK, tm * C::BM + (int)rank * 128);
 #pragma unroll
-                    for (int j = 0; j < 2; ++j)
-                        ptx::tma_load_2d_2cta(b_dst + j * C::kBChunkBytes, &map_b, full_leader,
-                                              tn * C::BN + (int)rank * 128 + j * 64, kb * C::BK);
+                    for (int u = 0; u < C::kSubK; ++u) {
+                        ptx::tma_load_2d_2cta(a_dst + u * C::kASubBytes, &map_a, full_leader, kb * C::BK + u * 64,
+                                              tm * C::BM + (int)rank * 128);
+#pragma unroll
+                        for (int j = 0; j < 2; ++j)
+                            ptx::tma_load_2d_2cta(b_dst + u * C::kBSubBytes + j * C::kBChunkBytes, &map_b, full_leader,
+                                                  tn * C::BN + (int)rank * 128 + j * 64, kb * C::BK + u * 64);
+                    }
                     if (++s == C::kStages) { s = 0; ph ^= 1; }
                 }
             }
@@ -240,7 +254,8 @@ gemm_umma2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     ptx::umma_bf16_2cta(d_tmem, desc(a_lo), desc(b_lo), idesc, kb != w.kb0);
 #pragma unroll
                     for (int k4 = 1; k4 < C::BK / 16; ++k4)
-                        ptx::umma_bf16_2cta_acc(d_tmem, desc(a_lo + 2 * k4), desc(b_lo + 128 * k4), idesc);
+                        ptx::umma_bf16_2cta_acc(d_tmem, desc(a_lo + (k4 / 4) * (C::kASubBytes >> 4) + 2 * (k4 % 4)),
+                                                desc(b_lo + (k4 / 4) * (C::kBSubBytes >> 4) + 128 * (k4 % 4)), idesc);
                     ptx::umma_commit_2cta(&sh->empty[s]);    // both CTAs: stage reusable once these MMAs have read it
                     if (++s == C::kStages) { s = 0; ph ^= 1; }
                 }
