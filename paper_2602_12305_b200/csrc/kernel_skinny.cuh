@@ -362,21 +362,24 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         if (lane == 0) {
             const uint64_t pol_stream = ptx::policy_evict_first();   // B is read exactly once
             const uint64_t pol_keep = ptx::policy_evict_last();      // A is re-read by every CTA
+            // ring positions and phases are carried along and wrapped by comparison: the issuing
+            // lanes are the critical path of this kernel, and a division per stage shows
             uint32_t it = 0, ait = 0;
+            int s = 0, sa = 0;
+            uint32_t ph = 0;
             bool ok = true;
             int site = 0;
             for (int tc = rect.t0; tc < rect.t1 && ok; tc += C::kAcc) {
                 const int nt = min(C::kAcc, rect.t1 - tc);
                 for (int kb = rect.kb0; kb < rect.kb1 && ok; ++kb, ++ait) {
-                    const int sa = ait % kAStagesRt;
                     ptx::mbar_arrive_expect_tx(&sh->a_full[sa], C::kABytes);
 #pragma unroll
                     for (int u = 0; u < C::kSub; ++u)
                         ptx::tma_load_2d_hint(aring + sa * C::kABytes + u * C::kASubBytes, &map_a, &sh->a_full[sa],
                                               kb * C::BK + u * 64, 0, pol_keep);
+                    if (++sa == kAStagesRt) sa = 0;
                     for (int j = 0; j < nt; ++j, ++it) {
-                        const int s = it % kStagesRt;
-                        if (sh->abort || (site = 1, !ptx::mbar_wait(&sh->empty[s], ((it / kStagesRt) & 1) ^ 1))) { ok = false; break; }
+                        if (sh->abort || (site = 1, !ptx::mbar_wait(&sh->empty[s], ph ^ 1))) { ok = false; break; }
                         uint8_t* b_dst = ring + s * C::kBBytes;
                         ptx::mbar_arrive_expect_tx(&sh->full[s], C::kBBytes);
 #pragma unroll
@@ -386,6 +389,7 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                             ptx::tma_load_2d_hint(b_dst + u * C::kBSubBytes + C::kBChunkBytes, &map_b, &sh->full[s],
                                                   (tc + j) * C::BN + 64, kb * C::BK + u * 64, pol_stream);
                         }
+                        if (++s == kStagesRt) { s = 0; ph ^= 1; }
                     }
                 }
             }
@@ -414,7 +418,17 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         if (lane == 0) {
             constexpr uint32_t idesc = ptx::umma_idesc_bf16(C::BN, MP, /*a_mn_major=*/true, /*b_mn_major=*/false);
             const int w = warp == 1 ? 0 : 1;                  // this lane takes the K steps w, w + kIssuers, ...
+            // Lean loop: ring positions and phases wrap by comparison (no division per stage), the
+            // abort flag is read once per K block, and the shared-memory descriptors are a constant
+            // high word plus a low word (start address in 16-byte units | leading offset << 16) that
+            // moves by constants from step to step.
+            constexpr uint32_t kDescHi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);   // stride 1024 B, version 1, 128-B swizzle
+            auto desc = [](uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; };
+            const uint32_t b_lo0 = ((ring_base & 0x3FFFFu) >> 4) | ((uint32_t)(C::kBChunkBytes >> 4) << 16);   // tiles of B (MMA "A")
+            const uint32_t a_lo0 = ((aring_base & 0x3FFFFu) >> 4) | ((16u >> 4) << 16);                          // tiles of A (MMA "B")
             uint32_t it = 0, ait = 0, chunk_it = 0;
+            int s = 0, sa = 0;
+            uint32_t ph = 0, pha = 0;
             bool ok = true;
             int site = 0;
             for (int tc = rect.t0; tc < rect.t1 && ok; tc += C::kAcc, ++chunk_it) {
@@ -423,25 +437,23 @@ gemm_skinny_umma_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 if (sh->abort || (site = 2, !ptx::mbar_wait(&sh->tmem_empty[half], ((chunk_it >> 1) & 1) ^ 1))) { ok = false; break; }
                 ptx::tcgen05_fence_after_sync();
                 for (int kb = rect.kb0; kb < rect.kb1 && ok; ++kb, ++ait) {
-                    const int sa = ait % kAStagesRt;
-                    if (sh->abort || (site = 3, !ptx::mbar_wait(&sh->a_full[sa], (ait / kAStagesRt) & 1))) { ok = false; break; }
-                    const uint32_t a_addr = aring_base + sa * C::kABytes;            // tile of A
+                    if (sh->abort || (site = 3, !ptx::mbar_wait(&sh->a_full[sa], pha))) { ok = false; break; }
+                    const uint32_t a_lo = a_lo0 + (uint32_t)sa * (uint32_t)(C::kABytes >> 4);
+                    if (++sa == kAStagesRt) { sa = 0; pha ^= 1; }
                     for (int j = 0; j < nt; ++j, ++it) {
-                        const int s = it % kStagesRt;
-                        if (sh->abort || (site = 4, !ptx::mbar_wait(&sh->full[s], (it / kStagesRt) & 1))) { ok = false; break; }
+                        if ((site = 4, !ptx::mbar_wait(&sh->full[s], ph))) { ok = false; break; }
                         ptx::tcgen05_fence_after_sync();
-                        const uint32_t b_addr = ring_base + s * C::kBBytes;          // tile of B
+                        const uint32_t b_lo = b_lo0 + (uint32_t)s * (uint32_t)(C::kBBytes >> 4);
                         const uint32_t d_tmem = tmem_base + skinny_acc_col<MP, SUB>(w, half, j);
 #pragma unroll
                         for (int q = 0; q < C::BK / 16 / C::kIssuers; ++q) {
                             const int k4 = q * C::kIssuers + w;
-                            const uint64_t da = ptx::umma_smem_desc(b_addr + (k4 / 4) * C::kBSubBytes + (k4 % 4) * 2048,
-                                                                    C::kBChunkBytes, 1024);
-                            const uint64_t db = ptx::umma_smem_desc(a_addr + (k4 / 4) * C::kASubBytes + (k4 % 4) * 32,
-                                                                    16, 1024);
+                            const uint64_t da = desc(b_lo + (uint32_t)((k4 / 4) * (C::kBSubBytes >> 4) + (k4 % 4) * (2048 >> 4)));
+                            const uint64_t db = desc(a_lo + (uint32_t)((k4 / 4) * (C::kASubBytes >> 4) + (k4 % 4) * (32 >> 4)));
                             ptx::umma_bf16(d_tmem, da, db, idesc, (kb != rect.kb0) || (q != 0));
                         }
                         ptx::umma_commit(&sh->empty[s]);
+                        if (++s == kStagesRt) { s = 0; ph ^= 1; }
                     }
                 }
                 if (ok) ptx::umma_commit(&sh->tmem_full[half]);
