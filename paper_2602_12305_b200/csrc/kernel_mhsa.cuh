@@ -174,58 +174,66 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             constexpr uint32_t idesc_o = ptx::umma_idesc_bf16(C::BQ, DK, false, true);        // P K-major, V MN-major
             bool ok = true;
             int site = 0;
-            // S_t = Q_t K_j^T, contraction over d_k in steps of 16 (32 bytes inside a 128-byte row)
-            auto issue_s = [&](int t, int j) {
-                const uint32_t q_addr = data_base + t * C::kTileBytes;
-                const uint32_t k_addr = data_base + C::kOffK + (j % C::kKSlots) * C::kTileBytes;
+            // Lean issuing loop (this lane is on the critical path): shared-memory descriptors are a
+            // constant high word plus a low word (start address in 16-byte units | leading offset
+            // << 16) advanced by constants; ring slots and phases wrap by comparison; the abort flag
+            // is read once per block.
+            constexpr uint32_t kDescHi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);   // stride 1024 B, version 1, 128-B swizzle
+            auto desc = [](uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; };
+            auto lo_k = [&](uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | ((16u >> 4) << 16); };                          // K-major
+            auto lo_mn = [&](uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | ((uint32_t)(C::kChunkBytes >> 4) << 16); };    // MN-major
+            const uint32_t q_lo = lo_k(data_base + t * C::kTileBytes);
+            const uint32_t p_lo = lo_k(data_base + C::kOffP + t * C::kPBytes);
+            const uint32_t k_lo0 = lo_k(data_base + C::kOffK), v_lo0 = lo_mn(data_base + C::kOffV);
+            const uint32_t d_s = tmem_base + C::kColS + t * C::BKV, d_o = tmem_base + C::kColO + t * DK;
+            const uint32_t p_tmem = tmem_base + C::kColP + t * 64;
+            // S_t = Q_t K^T, contraction over d_k in steps of 16 (32 bytes inside a 128-byte row)
+            auto issue_s = [&](uint32_t k_lo) {
 #pragma unroll
                 for (int ks = 0; ks < DK / 16; ++ks) {
-                    const uint32_t off = (ks >> 2) * C::kChunkBytes + (ks & 3) * 32;
-                    ptx::umma_bf16(tmem_base + C::kColS + t * C::BKV, ptx::umma_smem_desc(q_addr + off, 16, 1024),
-                                   ptx::umma_smem_desc(k_addr + off, 16, 1024), idesc_s, ks != 0);
+                    const uint32_t off = (uint32_t)(((ks >> 2) * C::kChunkBytes + (ks & 3) * 32) >> 4);
+                    ptx::umma_bf16(d_s, desc(q_lo + off), desc(k_lo + off), idesc_s, ks != 0);
                 }
                 ptx::umma_commit(&sh->s_full[t]);
             };
-            // O_t (+)= P_t V_j, contraction over the 128 keys in steps of 16 (16 rows of V)
-            auto issue_pv = [&](int t, int j) {
-                const uint32_t p_addr = data_base + C::kOffP + t * C::kPBytes;
-                const uint32_t v_addr = data_base + C::kOffV + (j % C::kVSlots) * C::kTileBytes;
+            // O_t (+)= P_t V, contraction over the 128 keys in steps of 16 (16 rows of V)
+            auto issue_pv = [&](uint32_t v_lo, bool first) {
 #pragma unroll
                 for (int ks = 0; ks < C::BKV / 16; ++ks) {
-                    const uint32_t p_off = (ks >> 2) * C::kChunkBytes + (ks & 3) * 32;
+                    const uint32_t p_off = (uint32_t)(((ks >> 2) * C::kChunkBytes + (ks & 3) * 32) >> 4);
                     if (C::kPInTmem)
-                        ptx::umma_bf16_tmem_a(tmem_base + C::kColO + t * DK, tmem_base + C::kColP + t * 64 + ks * 8,
-                                              ptx::umma_smem_desc(v_addr + ks * 2048, C::kChunkBytes, 1024), idesc_o,
-                                              j != 0 || ks != 0);
+                        ptx::umma_bf16_tmem_a(d_o, p_tmem + ks * 8, desc(v_lo + (uint32_t)(ks * (2048 >> 4))), idesc_o, !first || ks != 0);
                     else
-                        ptx::umma_bf16(tmem_base + C::kColO + t * DK, ptx::umma_smem_desc(p_addr + p_off, 16, 1024),
-                                       ptx::umma_smem_desc(v_addr + ks * 2048, C::kChunkBytes, 1024), idesc_o,
-                                       j != 0 || ks != 0);
+                        ptx::umma_bf16(d_o, desc(p_lo + p_off), desc(v_lo + (uint32_t)(ks * (2048 >> 4))), idesc_o, !first || ks != 0);
                 }
                 ptx::umma_commit(&sh->pv_done[t]);
             };
-            auto k_ready = [&](int j) { return ptx::mbar_wait(&sh->k_full[j % C::kKSlots], (j / C::kKSlots) & 1); };
-            auto v_ready = [&](int j) { return ptx::mbar_wait(&sh->v_full[j % C::kVSlots], (j / C::kVSlots) & 1); };
-            if (sh->abort || (site = 3, !ptx::mbar_wait(&sh->q_full, 0)) || (site = 4, !k_ready(0))) ok = false;
+            int ks_slot = 0, vs_slot = 0;                 // ring slots of K block j + 1 and of V block j
+            uint32_t k_ph = 0, v_ph = 0;
+            if (sh->abort || (site = 3, !ptx::mbar_wait(&sh->q_full, 0)) || (site = 4, !ptx::mbar_wait(&sh->k_full[0], 0))) ok = false;
             if (ok) {
                 ptx::tcgen05_fence_after_sync();
-                issue_s(t, 0);
+                issue_s(k_lo0);
                 ptx::umma_commit(&sh->k_empty[0]);
             }
+            if (++ks_slot == C::kKSlots) { ks_slot = 0; k_ph ^= 1; }
             for (int j = 0; ok && j < nblk; ++j) {
+                if (sh->abort) { ok = false; break; }
                 if (j + 1 < nblk) {
                     // the scores of block j + 1 as soon as the softmax threads hold block j in registers
-                    if (sh->abort || (site = 4, !k_ready(j + 1))) { ok = false; break; }
-                    if (sh->abort || (site = 6, !ptx::mbar_wait(&sh->s_free[t], j & 1))) { ok = false; break; }
+                    if ((site = 4, !ptx::mbar_wait(&sh->k_full[ks_slot], k_ph))) { ok = false; break; }
+                    if ((site = 6, !ptx::mbar_wait(&sh->s_free[t], j & 1))) { ok = false; break; }
                     ptx::tcgen05_fence_after_sync();
-                    issue_s(t, j + 1);
-                    ptx::umma_commit(&sh->k_empty[(j + 1) % C::kKSlots]);
+                    issue_s(k_lo0 + (uint32_t)ks_slot * (uint32_t)(C::kTileBytes >> 4));
+                    ptx::umma_commit(&sh->k_empty[ks_slot]);
+                    if (++ks_slot == C::kKSlots) { ks_slot = 0; k_ph ^= 1; }
                 }
-                if (sh->abort || (site = 5, !v_ready(j))) { ok = false; break; }
-                if (sh->abort || (site = 7, !ptx::mbar_wait(&sh->p_full[t], j & 1))) { ok = false; break; }
+                if ((site = 5, !ptx::mbar_wait(&sh->v_full[vs_slot], v_ph))) { ok = false; break; }
+                if ((site = 7, !ptx::mbar_wait(&sh->p_full[t], j & 1))) { ok = false; break; }
                 ptx::tcgen05_fence_after_sync();
-                issue_pv(t, j);
-                ptx::umma_commit(&sh->v_empty[j % C::kVSlots]);
+                issue_pv(v_lo0 + (uint32_t)vs_slot * (uint32_t)(C::kTileBytes >> 4), j == 0);
+                ptx::umma_commit(&sh->v_empty[vs_slot]);
+                if (++vs_slot == C::kVSlots) { vs_slot = 0; v_ph ^= 1; }
             }
             if (!ok) {
                 report_timeout(status, site);
