@@ -47,8 +47,8 @@ FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel,
 # from the ncu captures summarised under profiles/; None = not captured for the current kernel.
-NCU_TRAFFIC_BYTES = {"c1": 545792, "c2": 138099712, "c3": 121378816, "c4": 107639552, "c5": 4376021872,
-                     "sum": 272239616, "dot": 540065280, "mse": None, "a2": 254612736, "a3": 117895168}
+NCU_TRAFFIC_BYTES = {"c1": 545792, "c2": 138099712, "c3": 121091072, "c4": 107639552, "c5": 4376021872,
+                     "sum": 272239616, "dot": 540065280, "mse": None, "a2": 254764032, "a3": 117721344}
 
 
 def load_peaks():
@@ -516,7 +516,7 @@ def main():
                 r = main_res
             else:
                 # keep each region near a quarter of a second, but never more than --steps
-                guess_ms = {"c1": 545792.01, "c2": 0.025, "c3": 121378816.025, "c4": 107639552.12, "c5": 4376021872.8}[name]
+                guess_ms = {"c1": 545792.01, "c2": 0.025, "c3": 121091072.025, "c4": 107639552.12, "c5": 4376021872.8}[name]
                 k = max(10, min(args.steps, int(250.0 / guess_ms)))
                 r = measure(handle, name, args, sampler, device, peaks, peak_src, k, args.warmup)
             c = r["case"]
