@@ -356,6 +356,8 @@ def run_reference(args):
 def workload_config(case, name, variant):
     cfg = {"workload": f"{name}: {'fp32' if case.dtype == synth.F32 else 'bf16'} {case.M}x{case.N}x{case.K} "
                        f"bias + {['none', 'ReLU', 'GELU(tanh)'][case.act]}",
+           "arithmetic": "fp32 products and sums on the FMA pipes" if case.dtype == synth.F32
+                         else "exact bf16 products, fp32 accumulation, one rounding to bf16 at the store",
            "M": case.M, "N": case.N, "K": case.K,
            "l2": "consecutive steps use different buffer sets; one round over the sets moves >= 4 x L2"}
     if variant is not None:
@@ -536,7 +538,7 @@ def main():
 
     line = {"metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": region_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32" if case.dtype == synth.F32 else "bf16 inputs, f32 accumulate", "data": "synthetic",
+            "dtype": "f32" if case.dtype == synth.F32 else "bf16", "data": "synthetic",
             "config": workload_config(case, args.workload, main_res["variant"]),
             "tflops": case.flops / 1e12 * world / (region_ms / args.steps / 1e3),
             "gbs": case.algorithmic_bytes / 1e9 * world / (region_ms / args.steps / 1e3),
