@@ -189,13 +189,13 @@ __host__ __device__ __forceinline__ SkinnyRect skinny_rect(const SkinnyPlan& p, 
 // scratch can hold.  With unit_us <= 0 the cost of a plan is the largest rectangle area
 // (K blocks x column tiles) any CTA has to stream, ties going to fewer bands.  With
 // unit_us > 0 (the time one CTA needs to stream one unit at the per-SM rate) the cost is an
-// estimated run time, fitted to measurements on B200: a CTA streams at most about 58 GB/s,
-// all of them together at most about 6.5 TB/s (= 112 CTAs' worth), the two limits combine
-// like a 4-norm, and any split along K costs about 2.5 us for the partial-tile round trip.
-// So 112 whole tiles on 112 SMs beat a perfectly balanced two-band plan for a 118 MB
-// problem, while a 470 MB problem is better off balanced.
+// estimated run time, fitted to measurements on B200: a CTA streams at most at its own rate
+// (unit_us per unit), all of them together at most `dram_ctas` CTAs' worth of that (HBM), the
+// two limits combine like a 4-norm, and any split along K costs about 2.5 us for the
+// partial-tile round trip.  So 112 whole tiles on 112 SMs beat a perfectly balanced two-band
+// plan, while 64 tiles are better off cut into three bands on all SMs.
 inline SkinnyPlan make_skinny_plan(int64_t tiles, int64_t kblocks, int num_sms, int64_t max_slots,
-                                   double unit_us = 0.0) {
+                                   double unit_us = 0.0, double dram_ctas = 112.0) {
     const int64_t T = tiles, KB = kblocks;
     SkinnyPlan best;
     best.T = (int)T;
@@ -211,7 +211,7 @@ inline SkinnyPlan make_skinny_plan(int64_t tiles, int64_t kblocks, int num_sms, 
     auto estimate = [&](int64_t area, int nb) -> double {
         if (unit_us <= 0.0) return (double)area;
         const double t_sm = (double)area * unit_us;
-        const double t_dram = (double)(T * KB) * unit_us / 112.0;
+        const double t_dram = (double)(T * KB) * unit_us / dram_ctas;
         const double t = sqrt(sqrt(t_sm * t_sm * t_sm * t_sm + t_dram * t_dram * t_dram * t_dram));
         return t + (nb > 1 ? 2.5 : 0.0);
     };

@@ -289,9 +289,15 @@ optiml_status_t launch_skinny_cfg(optiml_handle_t h, const void* A, const void* 
     const CUtensorMap* mb = get_map(h, B, (uint64_t)K, (uint64_t)N, 64, 64);
     if (!ma || !mb) return OPTIML_ERR_CUDA;
     const int64_t max_slots = kPartialBytes / (C::kSlotFloats * sizeof(float));
-    // one unit = one K block of one column tile; a CTA streams it at about 58 GB/s
-    const double unit_us = (double)(C::kBBytes + C::kABytes) / 58.0e3;
-    const SkinnyPlan plan = make_skinny_plan(ceil_div64(N, C::BN), ceil_div64(K, C::BK), h->num_sms, max_slots, unit_us);
+    // one unit = one K block of one column tile; with two MMA lanes a CTA streams it at about 110 GB/s,
+    // all CTAs together at about 7 TB/s (measured: 16 x 14336 x 16384 as 112 whole tiles 67 us = 7.0 TB/s,
+    // as two balanced bands on 148 CTAs 76 us; 8 x 28672 x 4096 as one band on 148 CTAs 37.6 us, as two
+    // bands 46.7 us; 16 x 8192 x 8192 as three bands 22.9 us, as 64 whole tiles 26.3 us)
+    constexpr double kCtaGBs = 110.0, kAllGBs = 7000.0;
+    const double unit_us = (double)(C::kBBytes + C::kABytes) / (kCtaGBs * 1e3);
+    const SkinnyPlan plan = make_skinny_plan(ceil_div64(N, C::BN), ceil_div64(K, C::BK), h->num_sms, max_slots, unit_us,
+                                             kAllGBs / kCtaGBs);
+    if (h->log) fprintf(stderr, "[optiml] skinny plan: G=%d S=%d k_split=%d G1=%d k_mid=%d G2=%d bands=%d\n", plan.G, plan.S, plan.k_split, plan.G1, plan.k_mid, plan.G2, plan.nbands);
     SkinnyTune tune;
     const int64_t want = h->options[OPTIML_OPT_SKINNY_RING_STAGES];
     // default depth: all that fit, except three 192-row stages at M <= 16 (measured on 16 x 14336 x 4096
