@@ -20,7 +20,7 @@ guardrail sizes (1.0 spill, 0.5 registers, 0.5 work), rho_max (255, the hardware
 which state fixes the regime (the baseline's) and how a regression penalty enters (a term
 whose normalised change is negative is weighted by lambda instead of w).
 
-    python -m paper_2602_12305_b200.reward the benchmark spec CANDIDATE.md [T0_US T1_US]
+    python -m paper_2602_12305_b200.reward BEFORE_SUMMARY.md AFTER_SUMMARY.md [T0_US T1_US]
 
 reads two summaries in the format of this repository's profiles/ directory; the optional two
 numbers replace the run times measured under the profiler by times measured elsewhere (CUDA
