@@ -9,9 +9,10 @@
 // running maximum).  Warp roles:
 //   warp 0      TMA producer: the two 128-row Q tiles once, then K_0, V_0, K_1, V_1, ... through a ring
 //   warp 1      one lane issues the MMAs of query tile 0: S_0,j = Q_0 K_j^T and O_0 += P_0,j V_j
-//   warps 2-5   softmax + output for query tile 0 (one thread per query row = one TMEM lane)
-//   warps 6-9   the same for query tile 1
-//   warp 10     one lane issues the MMAs of query tile 1
+//   warp 2      one lane issues the MMAs of query tile 1
+//   warp 3      spare (completes the control warpgroup, which gives most of its registers away)
+//   warps 4-7   softmax + output for query tile 0 (one thread per query row = one TMEM lane)
+//   warps 8-11  the same for query tile 1
 // (One lane for both tiles was the bottleneck: a tcgen05.mma costs its issuer about 60 cycles and
 // every block also costs it six barrier waits, about 3000 cycles per key block in all, more than
 // the tensor pipe or the special-function unit need.)
@@ -47,7 +48,13 @@ struct MhsaCfg {
     // ring is double-buffered
     static constexpr int kKSlots = DK == 64 ? 3 : 1;
     static constexpr int kVSlots = DK == 64 ? 3 : 2;
-    static constexpr int kThreads = 352;                 // 11 warps: producer, MMA lane of tile 0, 8 softmax warps, MMA lane of tile 1
+    // 12 warps = 3 warpgroups: control (producer, MMA lane of tile 0, MMA lane of tile 1, one spare
+    // warp) and one softmax warpgroup per query tile.  Three warps share each SM sub-partition's
+    // 16384 registers, so a launch gives every thread 168; the control warpgroup hands most of
+    // its share back and the softmax warpgroups, which hold a whole row of scores, take it.
+    static constexpr int kThreads = 384;
+    static constexpr int kLaunchRegs = 168, kControlRegs = 48, kSoftmaxRegs = 224;
+    static_assert(128 * kControlRegs + 256 * kSoftmaxRegs <= kThreads * kLaunchRegs, "register shares exceed the launch's pool");
     static constexpr int kTmemCols = 512;                // S0, S1: 2 x 128; O0, O1: 2 x DK; P0, P1: 2 x 64
     static constexpr int kColS = 0, kColO = 256;
     // d_k = 64 leaves 128 columns of tensor memory for the probabilities (two bf16 per column),
@@ -123,129 +130,135 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const uint32_t tmem_base = sh->tmem_base;
     ptx::griddep_wait();
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            ptx::mbar_arrive_expect_tx(&sh->q_full, C::kQTiles * C::kTileBytes);
-            for (int t = 0; t < C::kQTiles; ++t)
-                for (int c = 0; c < C::kChunks; ++c)
-                    ptx::tma_load_2d(data + t * C::kTileBytes + c * C::kChunkBytes, &map_q, &sh->q_full,
-                                     head * DK + c * 64, q0 + t * C::BQ);
-            bool ok = true;
-            int site = 0, j = 0, done_k = 0, done_v = 0;
-            for (; ok && j < nblk; ++j) {
-                {
-                    const int s = j % C::kKSlots;
-                    const uint32_t ph = (j / C::kKSlots) & 1;
-                    if (sh->abort || (site = 1, !ptx::mbar_wait(&sh->k_empty[s], ph ^ 1))) { ok = false; break; }
-                    ptx::mbar_arrive_expect_tx(&sh->k_full[s], C::kTileBytes);
+    if (warp < 4) {
+        // control warpgroup: keeps few registers, the rest goes back to the pool
+        ptx::setmaxnreg_dec<C::kControlRegs>();
+        if (warp == 0) {
+            // ------------------------------------------------------------ TMA producer
+            if (lane == 0) {
+                ptx::mbar_arrive_expect_tx(&sh->q_full, C::kQTiles * C::kTileBytes);
+                for (int t = 0; t < C::kQTiles; ++t)
                     for (int c = 0; c < C::kChunks; ++c)
-                        ptx::tma_load_2d(data + C::kOffK + s * C::kTileBytes + c * C::kChunkBytes, &map_k, &sh->k_full[s],
-                                         head * DK + c * 64, j * C::BKV);
-                    done_k = j + 1;
+                        ptx::tma_load_2d(data + t * C::kTileBytes + c * C::kChunkBytes, &map_q, &sh->q_full,
+                                         head * DK + c * 64, q0 + t * C::BQ);
+                bool ok = true;
+                int site = 0, j = 0, done_k = 0, done_v = 0;
+                for (; ok && j < nblk; ++j) {
+                    {
+                        const int s = j % C::kKSlots;
+                        const uint32_t ph = (j / C::kKSlots) & 1;
+                        if (sh->abort || (site = 1, !ptx::mbar_wait(&sh->k_empty[s], ph ^ 1))) { ok = false; break; }
+                        ptx::mbar_arrive_expect_tx(&sh->k_full[s], C::kTileBytes);
+                        for (int c = 0; c < C::kChunks; ++c)
+                            ptx::tma_load_2d(data + C::kOffK + s * C::kTileBytes + c * C::kChunkBytes, &map_k, &sh->k_full[s],
+                                             head * DK + c * 64, j * C::BKV);
+                        done_k = j + 1;
+                    }
+                    {
+                        const int s = j % C::kVSlots;
+                        const uint32_t ph = (j / C::kVSlots) & 1;
+                        if (sh->abort || (site = 2, !ptx::mbar_wait(&sh->v_empty[s], ph ^ 1))) { ok = false; break; }
+                        ptx::mbar_arrive_expect_tx(&sh->v_full[s], C::kTileBytes);
+                        for (int c = 0; c < C::kChunks; ++c)
+                            ptx::tma_load_2d(data + C::kOffV + s * C::kTileBytes + c * C::kChunkBytes, &map_v, &sh->v_full[s],
+                                             head * DK + c * 64, j * C::BKV);
+                        done_v = j + 1;
+                    }
                 }
-                {
-                    const int s = j % C::kVSlots;
-                    const uint32_t ph = (j / C::kVSlots) & 1;
-                    if (sh->abort || (site = 2, !ptx::mbar_wait(&sh->v_empty[s], ph ^ 1))) { ok = false; break; }
-                    ptx::mbar_arrive_expect_tx(&sh->v_full[s], C::kTileBytes);
-                    for (int c = 0; c < C::kChunks; ++c)
-                        ptx::tma_load_2d(data + C::kOffV + s * C::kTileBytes + c * C::kChunkBytes, &map_v, &sh->v_full[s],
-                                         head * DK + c * 64, j * C::BKV);
-                    done_v = j + 1;
+                if (!ok) {
+                    report_timeout(status, site);
+                    sh->abort = 1;
+                    // copies already issued must land before the CTA may exit
+                    ptx::mbar_wait(&sh->q_full, 0);
+                    for (int b = 1; b <= C::kKSlots && b <= done_k; ++b)
+                        ptx::mbar_wait(&sh->k_full[(done_k - b) % C::kKSlots], ((done_k - b) / C::kKSlots) & 1);
+                    for (int b = 1; b <= C::kVSlots && b <= done_v; ++b)
+                        ptx::mbar_wait(&sh->v_full[(done_v - b) % C::kVSlots], ((done_v - b) / C::kVSlots) & 1);
                 }
             }
-            if (!ok) {
-                report_timeout(status, site);
-                sh->abort = 1;
-                // copies already issued must land before the CTA may exit
-                ptx::mbar_wait(&sh->q_full, 0);
-                for (int b = 1; b <= C::kKSlots && b <= done_k; ++b)
-                    ptx::mbar_wait(&sh->k_full[(done_k - b) % C::kKSlots], ((done_k - b) / C::kKSlots) & 1);
-                for (int b = 1; b <= C::kVSlots && b <= done_v; ++b)
-                    ptx::mbar_wait(&sh->v_full[(done_v - b) % C::kVSlots], ((done_v - b) / C::kVSlots) & 1);
-            }
-        }
-    } else if (warp == 1 || warp == 10) {
-        // ------------------------------------------------------------ MMA issuers, one per query tile
-        if (lane == 0) {
-            const int t = warp == 1 ? 0 : 1;
-            constexpr uint32_t idesc_s = ptx::umma_idesc_bf16(C::BQ, C::BKV, false, false);   // Q, K: both K-major
-            constexpr uint32_t idesc_o = ptx::umma_idesc_bf16(C::BQ, DK, false, true);        // P K-major, V MN-major
-            bool ok = true;
-            int site = 0;
-            // Lean issuing loop (this lane is on the critical path): shared-memory descriptors are a
-            // constant high word plus a low word (start address in 16-byte units | leading offset
-            // << 16) advanced by constants; ring slots and phases wrap by comparison; the abort flag
-            // is read once per block.
-            constexpr uint32_t kDescHi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);   // stride 1024 B, version 1, 128-B swizzle
-            auto desc = [](uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; };
-            auto lo_k = [&](uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | ((16u >> 4) << 16); };                          // K-major
-            auto lo_mn = [&](uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | ((uint32_t)(C::kChunkBytes >> 4) << 16); };    // MN-major
-            const uint32_t q_lo = lo_k(data_base + t * C::kTileBytes);
-            const uint32_t p_lo = lo_k(data_base + C::kOffP + t * C::kPBytes);
-            const uint32_t k_lo0 = lo_k(data_base + C::kOffK), v_lo0 = lo_mn(data_base + C::kOffV);
-            const uint32_t d_s = tmem_base + C::kColS + t * C::BKV, d_o = tmem_base + C::kColO + t * DK;
-            const uint32_t p_tmem = tmem_base + C::kColP + t * 64;
-            // S_t = Q_t K^T, contraction over d_k in steps of 16 (32 bytes inside a 128-byte row)
-            auto issue_s = [&](uint32_t k_lo) {
-#pragma unroll
-                for (int ks = 0; ks < DK / 16; ++ks) {
-                    const uint32_t off = (uint32_t)(((ks >> 2) * C::kChunkBytes + (ks & 3) * 32) >> 4);
-                    ptx::umma_bf16(d_s, desc(q_lo + off), desc(k_lo + off), idesc_s, ks != 0);
-                }
-                ptx::umma_commit(&sh->s_full[t]);
-            };
-            // O_t (+)= P_t V, contraction over the 128 keys in steps of 16 (16 rows of V)
-            auto issue_pv = [&](uint32_t v_lo, bool first) {
-#pragma unroll
-                for (int ks = 0; ks < C::BKV / 16; ++ks) {
-                    const uint32_t p_off = (uint32_t)(((ks >> 2) * C::kChunkBytes + (ks & 3) * 32) >> 4);
-                    if (C::kPInTmem)
-                        ptx::umma_bf16_tmem_a(d_o, p_tmem + ks * 8, desc(v_lo + (uint32_t)(ks * (2048 >> 4))), idesc_o, !first || ks != 0);
-                    else
-                        ptx::umma_bf16(d_o, desc(p_lo + p_off), desc(v_lo + (uint32_t)(ks * (2048 >> 4))), idesc_o, !first || ks != 0);
-                }
-                ptx::umma_commit(&sh->pv_done[t]);
-            };
-            int ks_slot = 0, vs_slot = 0;                 // ring slots of K block j + 1 and of V block j
-            uint32_t k_ph = 0, v_ph = 0;
-            if (sh->abort || (site = 3, !ptx::mbar_wait(&sh->q_full, 0)) || (site = 4, !ptx::mbar_wait(&sh->k_full[0], 0))) ok = false;
-            if (ok) {
-                ptx::tcgen05_fence_after_sync();
-                issue_s(k_lo0);
-                ptx::umma_commit(&sh->k_empty[0]);
-            }
-            if (++ks_slot == C::kKSlots) { ks_slot = 0; k_ph ^= 1; }
-            for (int j = 0; ok && j < nblk; ++j) {
-                if (sh->abort) { ok = false; break; }
-                if (j + 1 < nblk) {
-                    // the scores of block j + 1 as soon as the softmax threads hold block j in registers
-                    if ((site = 4, !ptx::mbar_wait(&sh->k_full[ks_slot], k_ph))) { ok = false; break; }
-                    if ((site = 6, !ptx::mbar_wait(&sh->s_free[t], j & 1))) { ok = false; break; }
+        } else if (warp == 1 || warp == 2) {
+            // ------------------------------------------------------------ MMA issuers, one per query tile
+            if (lane == 0) {
+                const int t = warp - 1;
+                constexpr uint32_t idesc_s = ptx::umma_idesc_bf16(C::BQ, C::BKV, false, false);   // Q, K: both K-major
+                constexpr uint32_t idesc_o = ptx::umma_idesc_bf16(C::BQ, DK, false, true);        // P K-major, V MN-major
+                bool ok = true;
+                int site = 0;
+                // Lean issuing loop (this lane is on the critical path): shared-memory descriptors are a
+                // constant high word plus a low word (start address in 16-byte units | leading offset
+                // << 16) advanced by constants; ring slots and phases wrap by comparison; the abort flag
+                // is read once per block.
+                constexpr uint32_t kDescHi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);   // stride 1024 B, version 1, 128-B swizzle
+                auto desc = [](uint32_t lo) { return ((uint64_t)kDescHi << 32) | lo; };
+                auto lo_k = [&](uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | ((16u >> 4) << 16); };                          // K-major
+                auto lo_mn = [&](uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | ((uint32_t)(C::kChunkBytes >> 4) << 16); };    // MN-major
+                const uint32_t q_lo = lo_k(data_base + t * C::kTileBytes);
+                const uint32_t p_lo = lo_k(data_base + C::kOffP + t * C::kPBytes);
+                const uint32_t k_lo0 = lo_k(data_base + C::kOffK), v_lo0 = lo_mn(data_base + C::kOffV);
+                const uint32_t d_s = tmem_base + C::kColS + t * C::BKV, d_o = tmem_base + C::kColO + t * DK;
+                const uint32_t p_tmem = tmem_base + C::kColP + t * 64;
+                // S_t = Q_t K^T, contraction over d_k in steps of 16 (32 bytes inside a 128-byte row)
+                auto issue_s = [&](uint32_t k_lo) {
+    #pragma unroll
+                    for (int ks = 0; ks < DK / 16; ++ks) {
+                        const uint32_t off = (uint32_t)(((ks >> 2) * C::kChunkBytes + (ks & 3) * 32) >> 4);
+                        ptx::umma_bf16(d_s, desc(q_lo + off), desc(k_lo + off), idesc_s, ks != 0);
+                    }
+                    ptx::umma_commit(&sh->s_full[t]);
+                };
+                // O_t (+)= P_t V, contraction over the 128 keys in steps of 16 (16 rows of V)
+                auto issue_pv = [&](uint32_t v_lo, bool first) {
+    #pragma unroll
+                    for (int ks = 0; ks < C::BKV / 16; ++ks) {
+                        const uint32_t p_off = (uint32_t)(((ks >> 2) * C::kChunkBytes + (ks & 3) * 32) >> 4);
+                        if (C::kPInTmem)
+                            ptx::umma_bf16_tmem_a(d_o, p_tmem + ks * 8, desc(v_lo + (uint32_t)(ks * (2048 >> 4))), idesc_o, !first || ks != 0);
+                        else
+                            ptx::umma_bf16(d_o, desc(p_lo + p_off), desc(v_lo + (uint32_t)(ks * (2048 >> 4))), idesc_o, !first || ks != 0);
+                    }
+                    ptx::umma_commit(&sh->pv_done[t]);
+                };
+                int ks_slot = 0, vs_slot = 0;                 // ring slots of K block j + 1 and of V block j
+                uint32_t k_ph = 0, v_ph = 0;
+                if (sh->abort || (site = 3, !ptx::mbar_wait(&sh->q_full, 0)) || (site = 4, !ptx::mbar_wait(&sh->k_full[0], 0))) ok = false;
+                if (ok) {
                     ptx::tcgen05_fence_after_sync();
-                    issue_s(k_lo0 + (uint32_t)ks_slot * (uint32_t)(C::kTileBytes >> 4));
-                    ptx::umma_commit(&sh->k_empty[ks_slot]);
-                    if (++ks_slot == C::kKSlots) { ks_slot = 0; k_ph ^= 1; }
+                    issue_s(k_lo0);
+                    ptx::umma_commit(&sh->k_empty[0]);
                 }
-                if ((site = 5, !ptx::mbar_wait(&sh->v_full[vs_slot], v_ph))) { ok = false; break; }
-                if ((site = 7, !ptx::mbar_wait(&sh->p_full[t], j & 1))) { ok = false; break; }
-                ptx::tcgen05_fence_after_sync();
-                issue_pv(v_lo0 + (uint32_t)vs_slot * (uint32_t)(C::kTileBytes >> 4), j == 0);
-                ptx::umma_commit(&sh->v_empty[vs_slot]);
-                if (++vs_slot == C::kVSlots) { vs_slot = 0; v_ph ^= 1; }
+                if (++ks_slot == C::kKSlots) { ks_slot = 0; k_ph ^= 1; }
+                for (int j = 0; ok && j < nblk; ++j) {
+                    if (sh->abort) { ok = false; break; }
+                    if (j + 1 < nblk) {
+                        // the scores of block j + 1 as soon as the softmax threads hold block j in registers
+                        if ((site = 4, !ptx::mbar_wait(&sh->k_full[ks_slot], k_ph))) { ok = false; break; }
+                        if ((site = 6, !ptx::mbar_wait(&sh->s_free[t], j & 1))) { ok = false; break; }
+                        ptx::tcgen05_fence_after_sync();
+                        issue_s(k_lo0 + (uint32_t)ks_slot * (uint32_t)(C::kTileBytes >> 4));
+                        ptx::umma_commit(&sh->k_empty[ks_slot]);
+                        if (++ks_slot == C::kKSlots) { ks_slot = 0; k_ph ^= 1; }
+                    }
+                    if ((site = 5, !ptx::mbar_wait(&sh->v_full[vs_slot], v_ph))) { ok = false; break; }
+                    if ((site = 7, !ptx::mbar_wait(&sh->p_full[t], j & 1))) { ok = false; break; }
+                    ptx::tcgen05_fence_after_sync();
+                    issue_pv(v_lo0 + (uint32_t)vs_slot * (uint32_t)(C::kTileBytes >> 4), j == 0);
+                    ptx::umma_commit(&sh->v_empty[vs_slot]);
+                    if (++vs_slot == C::kVSlots) { vs_slot = 0; v_ph ^= 1; }
+                }
+                if (!ok) {
+                    report_timeout(status, site);
+                    sh->abort = 1;
+                }
+                // nothing may be in flight on the tensor pipe when tensor memory is freed
+                ptx::umma_commit(&sh->drain);
+                ptx::mbar_wait(&sh->drain, 0);
             }
-            if (!ok) {
-                report_timeout(status, site);
-                sh->abort = 1;
-            }
-            // nothing may be in flight on the tensor pipe when tensor memory is freed
-            ptx::umma_commit(&sh->drain);
-            ptx::mbar_wait(&sh->drain, 0);
         }
     } else {
+        // softmax warpgroups: wait for their larger share (handed back above)
+        ptx::setmaxnreg_inc<C::kSoftmaxRegs>();
         // ------------------------------------------------------------ softmax + output, one thread per query row
-        const int t = (warp - 2) >> 2;                   // query tile of this warp group
+        const int t = (warp - 4) >> 2;                   // query tile of this warpgroup
         const int quarter = warp & 3;                    // TMEM lane quarter this warp may touch
         const int r = quarter * 32 + lane;               // row within the tile
         const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
@@ -284,7 +297,7 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 float a = __uint_as_float(v[c][0]);
 #pragma unroll
                 for (int i = 1; i < 32; i += 2)
-                    a = fmaxf(a, fmaxf(__uint_as_float(v[c][i]), __uint_as_float(v[c][(i + 1) & 31])));
+                    a = ptx::fmax3(a, __uint_as_float(v[c][i]), __uint_as_float(v[c][(i + 1) & 31]));
                 mx4[c] = a;
             }
             const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;

@@ -431,6 +431,11 @@ bool configure_kernels() {
     ok &= set_skinny(gemm_skinny_umma_kernel<128, 2>, SkinnyCfg<128, 2>::kSmemBytes);
     ok &= set_smem(mhsa_umma_kernel<64>, MhsaCfg<64>::kSmemBytes);
     ok &= set_smem(mhsa_umma_kernel<128>, MhsaCfg<128>::kSmemBytes);
+    // the attention kernel re-divides its registers between warpgroups and would wait forever
+    // if the launch handed out fewer than its shares add up to
+    cudaFuncAttributes fa;
+    ok = ok && cudaFuncGetAttributes(&fa, mhsa_umma_kernel<64>) == cudaSuccess && fa.numRegs >= MhsaCfg<64>::kLaunchRegs;
+    ok = ok && cudaFuncGetAttributes(&fa, mhsa_umma_kernel<128>) == cudaSuccess && fa.numRegs >= MhsaCfg<128>::kLaunchRegs;
     return ok;
 }
 

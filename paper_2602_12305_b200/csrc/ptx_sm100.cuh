@@ -240,6 +240,27 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
+// Register re-allocation between the warpgroups (four consecutive warps) of a CTA: every warp
+// of the warpgroup executes the same instruction.  `dec` hands registers back to the CTA's
+// pool (threads x registers per thread at launch), `inc` blocks until the pool can supply the
+// increase, so the shares of all warpgroups must add up to no more than the launch's total.
+template <int kRegs>
+__device__ __forceinline__ void setmaxnreg_dec() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
+template <int kRegs>
+__device__ __forceinline__ void setmaxnreg_inc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
+
+// Largest of three values in one instruction (issues at the rate of the two-input form:
+// measured 2 cycles per warp instruction and SM sub-partition for both).
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float y;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+    return y;
+}
+
 // ---------------------------------------------------------------- tcgen05.mma
 
 // D[tmem] (+)= A[smem] . B[smem]; bf16 inputs, fp32 accumulate; issued by ONE thread.
