@@ -66,6 +66,12 @@ struct MhsaCfg {
     static constexpr int kOffV = kOffK + kKSlots * kTileBytes;
     static constexpr int kSmemBytes = 256 + 1024 + kOffV + kVSlots * kTileBytes;
     static constexpr float kRescaleThreshold = 8.0f;     // log2 units
+    // Softmax warps overlap the round trips of their barrier waits with arithmetic (the abort flag
+    // is loaded beside the wait for the scores, the previous P V is polled once before the
+    // exponentials).  Measured at N = 16384 with 16 heads: d_k = 64 1375 -> 1267 us, but
+    // d_k = 128 1765 -> 2024 us: there the tensor pipe is the busy unit, K has a single slot, and
+    // softmax warps that arrive sooner make the two tiles' MMAs queue up in a worse order.
+    static constexpr bool kOverlapWaits = DK == 64;
 };
 
 struct MhsaShared {
@@ -270,8 +276,17 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         float2 l2[2] = {make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f)};
         bool ok = true;
         int site = 8;
+        // Every serial step of this loop is paid once per key block by a warp that has only one
+        // other warp on its sub-partition to hide behind, so the abort flag is read once per block
+        // (two more reads cost 5 % at d_k = 64); a wait whose partner has given up runs out by itself.
         for (int j = 0; j < nblk; ++j) {
-            bool got = !sh->abort && ptx::mbar_wait(&sh->s_full[t], j & 1);
+            bool got;
+            if (C::kOverlapWaits) {
+                const int aborted = sh->abort;           // its latency overlaps the wait's
+                got = ptx::mbar_wait(&sh->s_full[t], j & 1) && !aborted;
+            } else {
+                got = !sh->abort && ptx::mbar_wait(&sh->s_full[t], j & 1);
+            }
             got = __all_sync(0xffffffffu, got);
             if (!got) { ok = false; break; }
             ptx::tcgen05_fence_after_sync();
@@ -310,8 +325,7 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             bool prev_done = j == 0;                     // has P V of block j - 1 been waited for?
             if (__any_sync(0xffffffffu, raise)) {
                 // the accumulator is rescaled in place once the previous P V has finished
-                got = !sh->abort && ptx::mbar_wait(&sh->pv_done[t], (j - 1) & 1);
-                got = __all_sync(0xffffffffu, got);
+                got = __all_sync(0xffffffffu, ptx::mbar_wait(&sh->pv_done[t], (j - 1) & 1));
                 if (!got) { ok = false; site = 9; break; }
                 prev_done = true;
                 ptx::tcgen05_fence_after_sync();
@@ -331,6 +345,9 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 }
                 ptx::tmem_st_wait();
             }
+            // one early look at the previous P V (it has usually finished by now), so that the
+            // barrier's round trip overlaps the exponentials instead of following them
+            if (C::kOverlapWaits && !prev_done) prev_done = ptx::mbar_try_wait(&sh->pv_done[t], (j - 1) & 1);
             // probabilities relative to m_used: 2^(s * scale - m), packed to bf16 in place
             const float2 negm2 = make_float2(-m_used, -m_used);
 #pragma unroll
@@ -343,10 +360,9 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     v[c][i >> 1] = pack_bf16x2(e.x, e.y);
                 }
             }
-            if (!prev_done) {
+            if (!(C::kOverlapWaits ? __all_sync(0xffffffffu, prev_done) : prev_done)) {
                 // the previous P V still reads this tile's P buffer until it has finished
-                got = !sh->abort && ptx::mbar_wait(&sh->pv_done[t], (j - 1) & 1);
-                got = __all_sync(0xffffffffu, got);
+                got = __all_sync(0xffffffffu, ptx::mbar_wait(&sh->pv_done[t], (j - 1) & 1));
                 if (!got) { ok = false; site = 9; break; }
             }
             if (C::kPInTmem) {
