@@ -48,7 +48,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel,
 # from the ncu captures summarised under profiles/; None = not captured for the current kernel.
 NCU_TRAFFIC_BYTES = {"c1": 545792, "c2": 138099712, "c3": 121091072, "c4": 107639552, "c5": 4376021872,
-                     "sum": 272239616, "dot": 540065280, "mse": None, "a2": 254764032, "a3": 117721344}
+                     "sum": 272239616, "dot": 540065280, "mse": None, "a2": 250073088, "a3": 118124032}
 
 
 def load_peaks():
