@@ -29,6 +29,7 @@
 #ifndef OPTIML_H_
 #define OPTIML_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -143,7 +144,8 @@ optiml_status_t optiml_gemm_epilogue_host(optiml_handle_t h, const void* A_host,
  *
  * Returns OPTIML_ERR_UNSUPPORTED for M > 4, N > 65536 or N % 8 != 0 (nothing is
  * launched), ALIGNMENT for pointers that are not 16-byte aligned, ARCH on a device that
- * is not compute capability 10.0, INVALID_ARG / CUDA as elsewhere.
+ * is not compute capability 10.0, INVALID_ARG for a device index the process does not
+ * have (and as elsewhere), CUDA if a runtime call failed.
  *
  * The first call on each device looks up the scratch array's device address and the SM
  * count (host-side queries only) and keeps them for later calls; that first call
@@ -163,6 +165,31 @@ optiml_status_t optiml_gemv_noalloc(const void* A, const void* B, const void* bi
  * time-out has left Y undefined.
  */
 optiml_status_t optiml_get_last_status(optiml_handle_t h);
+
+/*
+ * Self-test of the failure path (host call, enqueues one tiny kernel on `stream`).  The paper
+ * prunes a candidate kernel that fails to run (Section 3.2, "Execution gate"); the counterpart
+ * here is that a kernel which gives up a bounded wait must REPORT it.  One CTA waits with the
+ * library's bounded wait, limited to `limit_cycles` SM cycles (1 .. 2e9), on a barrier that
+ * nobody signals, records the time-out in the handle's status word like every compute kernel
+ * would, and returns normally: no trap, no fault, the context stays usable.  Afterwards
+ * optiml_get_last_status returns OPTIML_ERR_TIMEOUT once (wait site 7 in the log), then OK.
+ * Returns INVALID_ARG for a NULL handle or a limit outside the range.
+ */
+optiml_status_t optiml_selftest_timeout(optiml_handle_t h, int64_t limit_cycles, void* stream);
+
+/*
+ * Failure injection for the library's own device allocations (host call; process-wide, not
+ * thread-safe; no counterpart in the paper).  While a hook is set, every allocation the library
+ * is about to make (handle scratch in optiml_create, staging buffers of
+ * optiml_gemm_epilogue_host) first calls hook(bytes, user); a non-zero return makes that
+ * allocation fail as if the device were out of memory, so the caller sees OPTIML_ERR_ALLOC.
+ * NULL removes the hook.  optiml_create frees whatever it had allocated before the failure;
+ * optiml_gemm_epilogue_host leaves the handle usable (the buffer that failed to grow is empty
+ * and is allocated again by the next call).
+ */
+typedef int (*optiml_alloc_hook_t)(size_t bytes, void* user);
+optiml_status_t optiml_set_alloc_hook(optiml_alloc_hook_t hook, void* user);
 
 /*
  * The K reduction on its own, over fp32 vectors of n elements (paper: Prompts appendix,

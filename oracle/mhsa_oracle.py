@@ -12,6 +12,10 @@ There is no mask and no output projection in the task.  Everything is fp64; the 
 definition exp(s_j) / sum_j exp(s_j), evaluated after subtracting the row maximum (which cancels
 exactly in the quotient and keeps exp in range).  bf16 tensors arrive as uint16 bit patterns and
 are widened exactly (a bf16 is the upper half of an fp32).
+
+The only library routine in the arithmetic is numpy's matrix product `@` (fp64), used for the two
+products per head; tests/test_mhsa_oracle.py replaces it by explicit loops over queries, keys and
+columns (an element-by-element brute force of the task's formula) and demands agreement.
 """
 from __future__ import annotations
 

@@ -37,6 +37,8 @@ EXPORTS = {
     "optiml_gemm_epilogue_host": (_ci, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _ci, _vp]),
     "optiml_gemv_noalloc": (_ci, [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _ci, _vp]),
     "optiml_get_last_status": (_ci, [_vp]),
+    "optiml_selftest_timeout": (_ci, [_vp, _i64, _vp]),
+    "optiml_set_alloc_hook": (_ci, [_vp, _vp]),
     "optiml_reduce_f32": (_ci, [_vp, _ci, _vp, _vp, _i64, _vp, _vp]),
     "optiml_mhsa": (_ci, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _ci, _vp]),
     "optiml_force_variant": (_ci, [_vp, _ci]),
@@ -119,6 +121,16 @@ def gemv_noalloc(A: torch.Tensor, B: torch.Tensor, bias: torch.Tensor | None, Y:
     _check(gemv_noalloc_raw(A.data_ptr(), B.data_ptr(), None if bias is None else bias.data_ptr(), Y.data_ptr(),
                             M, N, K, act, dev, st), "optiml_gemv_noalloc")
     return Y
+
+
+ALLOC_HOOK = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p)
+
+
+def set_alloc_hook(hook) -> None:
+    """optiml_set_alloc_hook: `hook` is an ALLOC_HOOK instance (keep a reference to it while it is
+    set) or None to remove it."""
+    lib = load_library()
+    _check(lib.optiml_set_alloc_hook(None if hook is None else ctypes.cast(hook, _vp), None), "optiml_set_alloc_hook")
 
 
 class Handle:
@@ -226,6 +238,10 @@ class Handle:
 
     def get_last_status(self) -> int:
         return self._lib.optiml_get_last_status(self._h)
+
+    def selftest_timeout(self, limit_cycles: int, stream: torch.cuda.Stream | None = None) -> int:
+        st = (stream or torch.cuda.current_stream(self.device)).cuda_stream
+        return self._lib.optiml_selftest_timeout(self._h, int(limit_cycles), st)
 
     def force_variant(self, variant: int):
         _check(self._lib.optiml_force_variant(self._h, int(variant)), "optiml_force_variant")

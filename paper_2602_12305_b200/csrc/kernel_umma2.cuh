@@ -33,13 +33,10 @@
 namespace optiml {
 
 struct Umma2Cfg {
-#ifndef OPTIML_UMMA2_SUBK
-#define OPTIML_UMMA2_SUBK 1
-#endif
-    // A stage holds kSubK sub-blocks of 64 k.  Every stage costs each issuing lane one barrier
-    // round trip, but three 128-k stages measured no better than six 64-k stages (4096^3: 103.4
-    // against 101.6 us; 8192 x 8192 x 16384: 1505 against 1491 us), so the finer ring stays.
-    static constexpr int kSubK = OPTIML_UMMA2_SUBK;
+    // A stage holds one 64-k block.  (Every stage costs each issuing lane one barrier round trip,
+    // but three 128-k stages measured no better than six 64-k stages: 4096^3 103.4 against
+    // 101.6 us, 8192 x 8192 x 16384 1505 against 1491 us.)
+    static constexpr int kSubK = 1;
     static constexpr int BM = 256, BN = 256, BK = 64 * kSubK, kStages = 6 / kSubK;   // tile of the CTA pair
     static constexpr int kASubBytes = 128 * 64 * 2;          // this CTA's 128 rows x 64 k of A: 16 KiB
     static constexpr int kABytes = kSubK * kASubBytes;

@@ -20,6 +20,7 @@
 #include "kernel_generic.cuh"
 #include "kernel_mhsa.cuh"
 #include "kernel_reduce.cuh"
+#include "kernel_selftest.cuh"
 #include "kernel_skinny.cuh"
 #include "kernel_umma.cuh"
 #include "kernel_umma2.cuh"
@@ -59,13 +60,36 @@ struct MapEntry {
 struct DeviceGuard {
     int prev = -1;
     bool switched = false;
+    bool ok = false;            // `dev` is the current device while the guard lives
     explicit DeviceGuard(int dev) {
-        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = (cudaSetDevice(dev) == cudaSuccess);
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        if (prev == dev) {
+            ok = true;
+            return;
+        }
+        ok = switched = (cudaSetDevice(dev) == cudaSuccess);
     }
     ~DeviceGuard() {
         if (switched) cudaSetDevice(prev);
     }
 };
+
+// Every device allocation of the library goes through here, so that a test can make the
+// n-th one fail (optiml_set_alloc_hook) without exhausting a GPU's memory.
+optiml_alloc_hook_t g_alloc_hook = nullptr;
+void* g_alloc_hook_user = nullptr;
+
+template <typename T>
+bool dev_alloc(T** p, size_t bytes) {
+    *p = nullptr;
+    if (g_alloc_hook && g_alloc_hook(bytes, g_alloc_hook_user) != 0) return false;
+    if (cudaMalloc(reinterpret_cast<void**>(p), bytes) != cudaSuccess) {
+        cudaGetLastError();
+        *p = nullptr;
+        return false;
+    }
+    return true;
+}
 
 }  // namespace
 
@@ -91,14 +115,18 @@ namespace {
 // ---------------------------------------------------------------- tensor maps
 
 // Row-major bf16 matrix [rows][cols] -> 2-D tiled map with a {box_cols, box_rows} box and
-// 128-byte swizzle (box_cols * 2 bytes == 128).  Cached by (pointer, shape, box).
-const CUtensorMap* get_map(optiml_handle_t h, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows,
-                           uint32_t box_cols) {
+// 128-byte swizzle (box_cols * 2 bytes == 128).  Cached by (pointer, shape, box).  The map is
+// COPIED into `out`, which the caller owns: a launch looks up two or three maps, and a miss on
+// a later lookup may recycle the very slot an earlier lookup of the same launch has hit.
+bool get_map(optiml_handle_t h, CUtensorMap* out, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows,
+             uint32_t box_cols) {
     for (int i = 0; i < kMapCache; ++i) {
-        MapEntry& e = h->maps[i];
+        const MapEntry& e = h->maps[i];
         if (e.valid && e.ptr == ptr && e.rows == rows && e.cols == cols && e.box_rows == box_rows &&
-            e.box_cols == box_cols)
-            return &e.map;
+            e.box_cols == box_cols) {
+            *out = e.map;
+            return true;
+        }
     }
     MapEntry& e = h->maps[h->next_map];
     h->next_map = (h->next_map + 1) % kMapCache;
@@ -110,14 +138,15 @@ const CUtensorMap* get_map(optiml_handle_t h, const void* ptr, uint64_t rows, ui
     CUresult r = h->encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box,
                            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return nullptr;
+    if (r != CUDA_SUCCESS) return false;
     e.ptr = ptr;
     e.rows = rows;
     e.cols = cols;
     e.box_rows = box_rows;
     e.box_cols = box_cols;
     e.valid = true;
-    return &e.map;
+    *out = e.map;
+    return true;
 }
 
 // ---------------------------------------------------------------- dispatcher
@@ -285,9 +314,9 @@ template <int MP, int SUB>
 optiml_status_t launch_skinny_cfg(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M,
                                   int N, int K, int act, cudaStream_t st) {
     using C = SkinnyCfg<MP, SUB>;
-    const CUtensorMap* ma = get_map(h, A, (uint64_t)M, (uint64_t)K, MP, 64);
-    const CUtensorMap* mb = get_map(h, B, (uint64_t)K, (uint64_t)N, 64, 64);
-    if (!ma || !mb) return OPTIML_ERR_CUDA;
+    CUtensorMap ma, mb;
+    if (!get_map(h, &ma, A, (uint64_t)M, (uint64_t)K, MP, 64) || !get_map(h, &mb, B, (uint64_t)K, (uint64_t)N, 64, 64))
+        return OPTIML_ERR_CUDA;
     const int64_t max_slots = kPartialBytes / (C::kSlotFloats * sizeof(float));
     // one unit = one K block of one column tile; with two MMA lanes a CTA streams it at about 110 GB/s,
     // all CTAs together at about 7 TB/s (measured: 16 x 14336 x 16384 as 112 whole tiles 67 us = 7.0 TB/s,
@@ -306,8 +335,8 @@ optiml_status_t launch_skinny_cfg(optiml_handle_t h, const void* A, const void* 
     tune.stages = want < 2 ? dflt : (want > C::kStages ? C::kStages : (int)want);
     tune.prefetch_early = (int)h->options[OPTIML_OPT_SKINNY_PREFETCH_EARLY];
     tune.late_trigger = h->options[OPTIML_OPT_SKINNY_LATE_TRIGGER] != 0;
-    launch_pdl(gemm_skinny_umma_kernel<MP, SUB>, dim3(plan.G), dim3(C::kThreads), C::smem_bytes(tune.stages), st, *ma,
-               *mb, (const __nv_bfloat16*)bias, (__nv_bfloat16*)Y, M, N, K, act, plan, tune, h->partials, h->counters,
+    launch_pdl(gemm_skinny_umma_kernel<MP, SUB>, dim3(plan.G), dim3(C::kThreads), C::smem_bytes(tune.stages), st, ma,
+               mb, (const __nv_bfloat16*)bias, (__nv_bfloat16*)Y, M, N, K, act, plan, tune, h->partials, h->counters,
                h->status);
     h->launches += 1;
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
@@ -335,29 +364,29 @@ optiml_status_t launch_skinny(optiml_handle_t h, const void* A, const void* B, c
 optiml_status_t launch_umma(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
                             int K, int act, cudaStream_t st) {
     using C = UmmaCfg;
-    const CUtensorMap* ma = get_map(h, A, (uint64_t)M, (uint64_t)K, C::BM, 64);
-    const CUtensorMap* mb = get_map(h, B, (uint64_t)K, (uint64_t)N, 64, 64);
-    const CUtensorMap* my = get_map(h, Y, (uint64_t)M, (uint64_t)N, 32, 64);
-    if (!ma || !mb || !my) return OPTIML_ERR_CUDA;
+    CUtensorMap ma, mb, my;
+    if (!get_map(h, &ma, A, (uint64_t)M, (uint64_t)K, C::BM, 64) || !get_map(h, &mb, B, (uint64_t)K, (uint64_t)N, 64, 64) ||
+        !get_map(h, &my, Y, (uint64_t)M, (uint64_t)N, 32, 64))
+        return OPTIML_ERR_CUDA;
     const UmmaPlan plan = make_umma_plan(M, N, K, h->num_sms);
     if ((size_t)plan.rem_tiles * plan.split * C::BM * C::BN * sizeof(float) > kPartialBytes) return OPTIML_ERR_UNSUPPORTED;
     const int grid = plan.grid;
     const __nv_bfloat16* bi = (const __nv_bfloat16*)bias;
     switch (act) {
     case OPTIML_ACT_RELU:
-        launch_pdl(gemm_umma_kernel<kActRelu>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
+        launch_pdl(gemm_umma_kernel<kActRelu>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, ma, mb, my, bi, M, N, K,
                    plan, h->partials, h->counters, h->status);
         break;
     case OPTIML_ACT_GELU_TANH:
-        launch_pdl(gemm_umma_kernel<kActGeluTanh>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
+        launch_pdl(gemm_umma_kernel<kActGeluTanh>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, ma, mb, my, bi, M, N, K,
                    plan, h->partials, h->counters, h->status);
         break;
     case OPTIML_ACT_SIGMOID:
-        launch_pdl(gemm_umma_kernel<kActSigmoid>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
+        launch_pdl(gemm_umma_kernel<kActSigmoid>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, ma, mb, my, bi, M, N, K,
                    plan, h->partials, h->counters, h->status);
         break;
     default:
-        launch_pdl(gemm_umma_kernel<kActNone>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
+        launch_pdl(gemm_umma_kernel<kActNone>, dim3(grid), dim3(C::kThreads), C::kSmemBytes, st, ma, mb, my, bi, M, N, K,
                    plan, h->partials, h->counters, h->status);
         break;
     }
@@ -368,10 +397,10 @@ optiml_status_t launch_umma(optiml_handle_t h, const void* A, const void* B, con
 optiml_status_t launch_umma2(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
                              int K, int act, cudaStream_t st) {
     using C = Umma2Cfg;
-    const CUtensorMap* ma = get_map(h, A, (uint64_t)M, (uint64_t)K, 128, 64);
-    const CUtensorMap* mb = get_map(h, B, (uint64_t)K, (uint64_t)N, 64, 64);
-    const CUtensorMap* my = get_map(h, Y, (uint64_t)M, (uint64_t)N, 32, 64);
-    if (!ma || !mb || !my) return OPTIML_ERR_CUDA;
+    CUtensorMap ma, mb, my;
+    if (!get_map(h, &ma, A, (uint64_t)M, (uint64_t)K, 128, 64) || !get_map(h, &mb, B, (uint64_t)K, (uint64_t)N, 64, 64) ||
+        !get_map(h, &my, Y, (uint64_t)M, (uint64_t)N, 32, 64))
+        return OPTIML_ERR_CUDA;
     const UmmaPlan plan = make_umma2_plan(M, N, K, h->num_sms);
     if ((size_t)plan.rem_tiles * plan.split * C::BM * C::BN * sizeof(float) > kPartialBytes) return OPTIML_ERR_UNSUPPORTED;
     if (2 * plan.rem_tiles > kNumCounters) return OPTIML_ERR_UNSUPPORTED;
@@ -379,19 +408,19 @@ optiml_status_t launch_umma2(optiml_handle_t h, const void* A, const void* B, co
     const __nv_bfloat16* bi = (const __nv_bfloat16*)bias;
     switch (act) {
     case OPTIML_ACT_RELU:
-        launch_pdl(gemm_umma2_kernel<kActRelu>, grid, dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
+        launch_pdl(gemm_umma2_kernel<kActRelu>, grid, dim3(C::kThreads), C::kSmemBytes, st, ma, mb, my, bi, M, N, K,
                    plan, h->partials, h->counters, h->status);
         break;
     case OPTIML_ACT_GELU_TANH:
-        launch_pdl(gemm_umma2_kernel<kActGeluTanh>, grid, dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N,
+        launch_pdl(gemm_umma2_kernel<kActGeluTanh>, grid, dim3(C::kThreads), C::kSmemBytes, st, ma, mb, my, bi, M, N,
                    K, plan, h->partials, h->counters, h->status);
         break;
     case OPTIML_ACT_SIGMOID:
-        launch_pdl(gemm_umma2_kernel<kActSigmoid>, grid, dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N,
+        launch_pdl(gemm_umma2_kernel<kActSigmoid>, grid, dim3(C::kThreads), C::kSmemBytes, st, ma, mb, my, bi, M, N,
                    K, plan, h->partials, h->counters, h->status);
         break;
     default:
-        launch_pdl(gemm_umma2_kernel<kActNone>, grid, dim3(C::kThreads), C::kSmemBytes, st, *ma, *mb, *my, bi, M, N, K,
+        launch_pdl(gemm_umma2_kernel<kActNone>, grid, dim3(C::kThreads), C::kSmemBytes, st, ma, mb, my, bi, M, N, K,
                    plan, h->partials, h->counters, h->status);
         break;
     }
@@ -443,13 +472,13 @@ template <int DK>
 optiml_status_t launch_mhsa_umma(optiml_handle_t h, const void* Q, const void* K, const void* V, void* Y, int N,
                                  int d_model, int heads, cudaStream_t st) {
     using C = MhsaCfg<DK>;
-    const CUtensorMap* mq = get_map(h, Q, (uint64_t)N, (uint64_t)d_model, 128, 64);
-    const CUtensorMap* mk = get_map(h, K, (uint64_t)N, (uint64_t)d_model, 128, 64);
-    const CUtensorMap* mv = get_map(h, V, (uint64_t)N, (uint64_t)d_model, 128, 64);
-    if (!mq || !mk || !mv) return OPTIML_ERR_CUDA;
+    CUtensorMap mq, mk, mv;
+    if (!get_map(h, &mq, Q, (uint64_t)N, (uint64_t)d_model, 128, 64) || !get_map(h, &mk, K, (uint64_t)N, (uint64_t)d_model, 128, 64) ||
+        !get_map(h, &mv, V, (uint64_t)N, (uint64_t)d_model, 128, 64))
+        return OPTIML_ERR_CUDA;
     const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)DK));
     const dim3 grid((unsigned)ceil_div64(N, C::kQTiles * C::BQ), (unsigned)heads);
-    launch_pdl(mhsa_umma_kernel<DK>, grid, dim3(C::kThreads), C::kSmemBytes, st, *mq, *mk, *mv, (__nv_bfloat16*)Y, N,
+    launch_pdl(mhsa_umma_kernel<DK>, grid, dim3(C::kThreads), C::kSmemBytes, st, mq, mk, mv, (__nv_bfloat16*)Y, N,
                d_model, scale_log2, h->status);
     h->launches += 1;
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
@@ -515,12 +544,11 @@ optiml_status_t optiml_create(optiml_handle_t* out, int device) {
     }
     h->encode = reinterpret_cast<encode_tiled_fn>(fn);
 
-    bool ok = cudaMalloc(&h->partials, kPartialBytes) == cudaSuccess;
-    ok = ok && cudaMalloc(&h->counters, kNumCounters * sizeof(unsigned int)) == cudaSuccess;
-    ok = ok && cudaMalloc(&h->status, sizeof(int)) == cudaSuccess;
+    bool ok = dev_alloc(&h->partials, kPartialBytes);
+    ok = ok && dev_alloc(&h->counters, kNumCounters * sizeof(unsigned int));
+    ok = ok && dev_alloc(&h->status, sizeof(int));
     if (!ok) {
-        cudaGetLastError();
-        optiml_destroy(h);
+        optiml_destroy(h);       // frees what was allocated before the failure
         return OPTIML_ERR_ALLOC;
     }
     ok = cudaMemset(h->counters, 0, kNumCounters * sizeof(unsigned int)) == cudaSuccess;
@@ -600,10 +628,7 @@ optiml_status_t optiml_gemm_epilogue_host(optiml_handle_t h, const void* A_host,
         cudaFree(h->stage[i]);
         h->stage[i] = nullptr;
         h->stage_bytes[i] = 0;
-        if (cudaMalloc(&h->stage[i], need[i]) != cudaSuccess) {
-            cudaGetLastError();
-            return OPTIML_ERR_ALLOC;
-        }
+        if (!dev_alloc(&h->stage[i], need[i])) return OPTIML_ERR_ALLOC;   // the handle stays usable; this buffer is empty
         h->stage_bytes[i] = need[i];
     }
     bool ok = cudaMemcpyAsync(h->stage[0], A_host, need[0], cudaMemcpyHostToDevice, st) == cudaSuccess;
@@ -633,6 +658,21 @@ optiml_status_t optiml_get_last_status(optiml_handle_t h) {
         cudaDeviceSynchronize();
         return OPTIML_ERR_TIMEOUT;
     }
+    return OPTIML_OK;
+}
+
+optiml_status_t optiml_selftest_timeout(optiml_handle_t h, int64_t limit_cycles, void* stream) {
+    if (!h || limit_cycles < 1 || limit_cycles > kSelftestMaxCycles) return OPTIML_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    launch_pdl(selftest_timeout_kernel, dim3(1), dim3(32), 0, static_cast<cudaStream_t>(stream), (long long)limit_cycles,
+               h->status);
+    h->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+optiml_status_t optiml_set_alloc_hook(optiml_alloc_hook_t hook, void* user) {
+    g_alloc_hook = hook;
+    g_alloc_hook_user = user;
     return OPTIML_OK;
 }
 
@@ -775,12 +815,21 @@ optiml_status_t optiml_gemv_noalloc(const void* A, const void* B, const void* bi
                                     int64_t K, optiml_act_t act, int device, void* stream) {
     if (!A || !B || !Y || M < 1 || N < 1 || K < 1 || K > INT32_MAX) return OPTIML_ERR_INVALID_ARG;
     if (act != OPTIML_ACT_NONE && act != OPTIML_ACT_RELU && act != OPTIML_ACT_GELU_TANH && act != OPTIML_ACT_SIGMOID) return OPTIML_ERR_INVALID_ARG;
-    if (device < 0 || device >= kNoAllocMaxDevices) return OPTIML_ERR_INVALID_ARG;
+    int device_count = 0;
+    if (cudaGetDeviceCount(&device_count) != cudaSuccess) {
+        cudaGetLastError();
+        return OPTIML_ERR_CUDA;
+    }
+    if (device < 0 || device >= device_count || device >= kNoAllocMaxDevices) return OPTIML_ERR_INVALID_ARG;
     // limits of the fixed scratch and of the kernel: refuse, never truncate
     if (M > 4 || N > kNoAllocMaxN || N % 8 != 0) return OPTIML_ERR_UNSUPPORTED;
     if (!(aligned16(A) && aligned16(B) && aligned16(bias) && aligned16(Y))) return OPTIML_ERR_ALIGNMENT;
 
     DeviceGuard guard(device);
+    if (!guard.ok) {
+        cudaGetLastError();
+        return OPTIML_ERR_CUDA;
+    }
     if (!g_noalloc_ptr[device]) {
         // One-time set-up on this device (it must be the current one here).  In host code the
         // name of a __device__ array is only a stand-in; the address a kernel may use comes
@@ -788,8 +837,10 @@ optiml_status_t optiml_gemv_noalloc(const void* A, const void* B, const void* bi
         int major = 0, minor = 0, sms = 0;
         if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
             cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, device) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+            cudaGetLastError();
             return OPTIML_ERR_CUDA;
+        }
         if (major != 10 || minor != 0) return OPTIML_ERR_ARCH;
         unsigned char* p = nullptr;
         if (cudaGetSymbolAddress((void**)&p, g_noalloc_scratch) != cudaSuccess || !p) {
@@ -797,7 +848,7 @@ optiml_status_t optiml_gemv_noalloc(const void* A, const void* B, const void* bi
             return OPTIML_ERR_CUDA;
         }
         g_noalloc_sms[device] = sms;
-        g_noalloc_ptr[device] = p;
+        g_noalloc_ptr[device] = p;       // published last: a non-null pointer means the SM count is set
     }
     unsigned char* base = g_noalloc_ptr[device];
     unsigned int* counters = reinterpret_cast<unsigned int*>(base);

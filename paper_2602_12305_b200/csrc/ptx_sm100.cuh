@@ -41,31 +41,30 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-__device__ __forceinline__ uint64_t global_timer_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-
 // Wait for the phase with the given parity to complete, but never forever: the SM's cycle
-// counter is checked every 64 failed polls and after kWaitLimitCycles (two to three seconds
-// at 1.3-1.97 GHz, far beyond any legitimate wait in these kernels) the wait gives up and
+// counter is checked every 64 failed polls and after `limit_cycles` the wait gives up and
 // returns false.  The caller then records a time-out in the handle's status word and leaves
 // through the common tear-down path.  (The cycle counter, not %globaltimer: the global timer
 // can be stepped from outside, while clock64 only ever counts this SM's cycles.  With the
 // global timer one time-out was reported in some 50 000 launches and never reproduced.)
-constexpr long long kWaitLimitCycles = 4000000000ll;
-
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t* bar, uint32_t parity, long long limit_cycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t i = 1;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 63u) == 0u) {
-            if (clock64() - t0 > kWaitLimitCycles) return false;
+            if (clock64() - t0 > limit_cycles) return false;
             __nanosleep(32);
         }
     }
+}
+
+// The limit every kernel uses: two to three seconds at 1.3-1.97 GHz, far beyond any legitimate
+// wait in these kernels.
+constexpr long long kWaitLimitCycles = 4000000000ll;
+
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    return mbar_wait_limit(bar, parity, kWaitLimitCycles);
 }
 
 // ---------------------------------------------------------------- programmatic dependent launch

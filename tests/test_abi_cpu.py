@@ -63,6 +63,17 @@ def test_null_arguments_are_rejected_before_any_cuda_call(lib):
     assert lib.optiml_launch_count(None) == -1
     assert lib.optiml_set_option(None, 0, 1) == binding.ERR_INVALID_ARG
     assert lib.optiml_get_option(None, 0) == -1
+    assert lib.optiml_selftest_timeout(None, 1000, None) == binding.ERR_INVALID_ARG
+    assert lib.optiml_reduce_f32(None, 0, 16, None, 1, 16, None) == binding.ERR_INVALID_ARG
+    assert lib.optiml_mhsa(None, 16, 16, 16, 16, 1, 1, 1, 1, None) == binding.ERR_INVALID_ARG
+
+
+def test_alloc_hook_can_be_set_and_removed_without_a_gpu(lib):
+    calls = []
+    cb = binding.ALLOC_HOOK(lambda nbytes, user: calls.append(nbytes) or 1)
+    binding.set_alloc_hook(cb)
+    binding.set_alloc_hook(None)
+    assert calls == []                      # setting a hook allocates nothing by itself
 
 
 @pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU behaviour")

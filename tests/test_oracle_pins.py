@@ -151,6 +151,23 @@ def test_gelu_tanh_is_the_tanh_form_not_erf():
     assert 1e-4 < d < 1e-3        # the tanh form differs from the erf form by a few 1e-4
 
 
+def test_gelu_tanh_stored_values():
+    """Golden values written with 50-digit decimal arithmetic (tests/golden/make_gelu_tanh_values.py):
+    G(0), G(+-0.5), G(+-1), G(+-2), G(+-3), G(+-6) and three more, to a few ulp of fp64."""
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "gelu_tanh_values.txt")
+    rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    assert len(rows) >= 11
+    for xs, gs in rows:
+        x, want = float(xs), float(gs)
+        got = oracle.act(x, GELU)
+        # the cancellation in 1 + tanh(u) for negative x costs absolute, not relative, accuracy
+        assert abs(got - want) <= 4e-16 * max(abs(x), 1e-3), (x, got, want)
+        # and through the whole function: K = 1, B = [1], no bias
+        y = run(enc([x], F32), enc([1.0], F32), None, 1, 1, 1, F32, GELU)
+        assert abs(y[0, 0] - want) <= 4e-16 * max(abs(x), 1e-3)
+
+
 def test_gelu_through_the_gemm():
     xs = np.array([-2.0, -1.0, -0.5, 0.5, 1.0, 2.0, 3.0])
     y = run(enc(xs[:, None], F32), enc([[1.0]], F32), None, len(xs), 1, 1, F32, GELU)

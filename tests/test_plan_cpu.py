@@ -9,9 +9,10 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 def test_skinny_schedule_selftest(tmp_path):
     exe = tmp_path / "plan_selftest"
-    src = os.path.join(ROOT, "paper_2602_12305_b200", "csrc", "plan_selftest.cu")
-    subprocess.run(["nvcc", "-std=c++17", "-O1", "-gencode", "arch=compute_100a,code=sm_100a", "-o", str(exe), src],
-                   check=True)
+    src = os.path.join(ROOT, "tests", "plan_selftest.cu")
+    inc = os.path.join(ROOT, "paper_2602_12305_b200", "csrc")
+    subprocess.run(["nvcc", "-std=c++17", "-O1", "-gencode", "arch=compute_100a,code=sm_100a", "-I", inc, "-o", str(exe),
+                    src], check=True)
     out = subprocess.run([str(exe)], capture_output=True, text=True)
     assert out.returncode == 0, out.stdout
     assert "0 failed" in out.stdout
