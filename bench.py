@@ -656,7 +656,8 @@ def workload_config(case, name, variant):
 
 # ---------------------------------------------------------------- the dispatcher's crossover table
 
-CROSSOVER_VARIANTS = ["gemv_splitk_stream", "skinny_streamk_tcgen05", "persistent_tcgen05", "persistent_tcgen05_cta_pair"]
+CROSSOVER_VARIANTS = ["gemv_splitk_stream", "skinny_streamk_tcgen05", "persistent_tcgen05", "persistent_tcgen05_cta_pair",
+                      "cluster_splitk_tcgen05_cta_pair"]
 
 
 def run_crossover(args):

@@ -16,13 +16,14 @@ F32, BF16 = 0, 1
 ACT_NONE, ACT_RELU, ACT_GELU_TANH, ACT_SIGMOID = 0, 1, 2, 3
 VARIANT_AUTO, VARIANT_GENERIC, VARIANT_F32_TILED, VARIANT_GEMV_SPLITK, VARIANT_SKINNY_UMMA, VARIANT_UMMA = -1, 0, 1, 2, 3, 4
 VARIANT_UMMA_2CTA = 5
-VARIANT_COUNT = 6
+VARIANT_UMMA_2CTA_STREAM = 6
+VARIANT_COUNT = 7
 
 REDUCE_SUM, REDUCE_DOT, REDUCE_MSE = 0, 1, 2
 
 (OPT_GEMV_PREFETCH_ROWS, OPT_SKINNY_STAGE_ROWS, OPT_SKINNY_RING_STAGES, OPT_SKINNY_PREFETCH_EARLY,
- OPT_SKINNY_LATE_TRIGGER) = range(5)
-OPT_COUNT = 5
+ OPT_SKINNY_LATE_TRIGGER, OPT_PAIR_SPLIT_MAX) = range(6)
+OPT_COUNT = 6
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ARCH, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(8)
 

@@ -52,7 +52,7 @@ struct Umma2Cfg {
 };
 
 // Same work split as make_umma_plan, over 256 x 256 tiles and CTA pairs.
-inline UmmaPlan make_umma2_plan(int64_t M, int64_t N, int64_t K, int num_sms) {
+inline UmmaPlan make_umma2_plan(int64_t M, int64_t N, int64_t K, int num_sms, int split_max = 8) {
     const int pairs = num_sms / 2;
     UmmaPlan p;
     p.tiles_m = (int)((M + Umma2Cfg::BM - 1) / Umma2Cfg::BM);
@@ -63,7 +63,7 @@ inline UmmaPlan make_umma2_plan(int64_t M, int64_t N, int64_t K, int num_sms) {
     int split = 1;
     if (r > 0) {
         split = (int)(pairs / r);
-        if (split > 8) split = 8;
+        if (split > split_max) split = split_max;
         if (split > p.num_kb * Umma2Cfg::kSubK / 4) split = p.num_kb * Umma2Cfg::kSubK / 4;   // at least 256 k per slice
         if (split > p.num_kb) split = p.num_kb;
         if (split < 1) split = 1;
@@ -80,20 +80,6 @@ inline UmmaPlan make_umma2_plan(int64_t M, int64_t N, int64_t K, int num_sms) {
     p.split = split;
     return p;
 }
-
-struct Umma2Shared {
-    uint64_t full[Umma2Cfg::kStages];      // used in the leader: bytes of both CTAs land here
-    uint64_t empty[Umma2Cfg::kStages];     // per CTA, signalled by the leader's commit
-    uint64_t tmem_full[2];                 // per CTA, signalled by the leader's commit
-    uint64_t tmem_empty[2];                // used in the leader: 256 epilogue threads arrive
-    uint64_t drain;
-    uint32_t tmem_base;
-    volatile int abort;
-    int last_flag;
-    int vote[4];
-};
-
-__device__ __forceinline__ void umma2_epi_bar_sync() { asm volatile("bar.sync 3, 128;" ::: "memory"); }
 
 // i-th work item of CTA pair `c`; tile coordinates in units of 256 x 256.
 __device__ __forceinline__ bool umma2_work_item(const UmmaPlan& p, int c, int i, UmmaWork& w) {
@@ -124,6 +110,20 @@ __device__ __forceinline__ bool umma2_work_item(const UmmaPlan& p, int c, int i,
     w.kb1 = (int)((int64_t)p.num_kb * (w.chunk + 1) / p.split);
     return true;
 }
+
+struct Umma2Shared {
+    uint64_t full[Umma2Cfg::kStages];      // used in the leader: bytes of both CTAs land here
+    uint64_t empty[Umma2Cfg::kStages];     // per CTA, signalled by the leader's commit
+    uint64_t tmem_full[2];                 // per CTA, signalled by the leader's commit
+    uint64_t tmem_empty[2];                // used in the leader: 256 epilogue threads arrive
+    uint64_t drain;
+    uint32_t tmem_base;
+    volatile int abort;
+    int last_flag;
+    int vote[4];
+};
+
+__device__ __forceinline__ void umma2_epi_bar_sync() { asm volatile("bar.sync 3, 128;" ::: "memory"); }
 
 template <int ACT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(Umma2Cfg::kThreads, 1)

@@ -24,6 +24,7 @@
 #include "kernel_skinny.cuh"
 #include "kernel_umma.cuh"
 #include "kernel_umma2.cuh"
+#include "kernel_umma2s.cuh"
 
 using namespace optiml;
 
@@ -43,7 +44,11 @@ constexpr int64_t kOptionDefaults[OPTIML_OPT_COUNT] = {
     /* SKINNY_RING_STAGES    */ 0,
     /* SKINNY_PREFETCH_EARLY */ 4,
     /* SKINNY_LATE_TRIGGER   */ 1,
+    /* PAIR_SPLIT_MAX        */ 8,
 };
+
+// Streaming rates the skinny kernel's schedule is costed with (see launch_skinny_cfg).
+constexpr double kSkinnyCtaGBs = 110.0, kSkinnyAllGBs = 7000.0;
 
 typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                     const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -108,6 +113,7 @@ struct optiml_handle_s {
     void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
     size_t stage_bytes[4] = {0, 0, 0, 0};
     int64_t options[OPTIML_OPT_COUNT];
+    int stream_clusters[2] = {0, 0};      // clusters of 2 and of 4 CTAs of the streaming pair kernel the device can hold at once
 };
 
 namespace {
@@ -153,7 +159,7 @@ bool get_map(optiml_handle_t h, CUtensorMap* out, const void* ptr, uint64_t rows
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
-bool variant_supports(int v, int64_t M, int64_t N, int64_t K, int dtype, bool al16) {
+bool variant_supports(optiml_handle_t h, int v, int64_t M, int64_t N, int64_t K, int dtype, bool al16) {
     switch (v) {
     case OPTIML_VARIANT_GENERIC:
         return true;
@@ -169,9 +175,40 @@ bool variant_supports(int v, int64_t M, int64_t N, int64_t K, int dtype, bool al
     case OPTIML_VARIANT_UMMA_2CTA:
         return dtype == OPTIML_BF16 && N % 8 == 0 && K % 8 == 0 && al16 &&
                ceil_div64(M, UmmaCfg::BM) * ceil_div64(N, UmmaCfg::BN) < (int64_t)1 << 31;
+    case OPTIML_VARIANT_UMMA_2CTA_STREAM:
+        // one cluster per 256 x 256 tile, all of them resident at once
+        return dtype == OPTIML_BF16 && N % 8 == 0 && K % 8 == 0 && al16 &&
+               ceil_div64(M, Umma2sCfg::BM) * ceil_div64(N, Umma2sCfg::BN) <= h->stream_clusters[0];
     default:
         return false;
     }
+}
+
+// K slices (CTA pairs per tile) of the streaming pair kernel: as many as the device can hold
+// clusters for, with at least four K blocks per slice.
+int stream_split(optiml_handle_t h, int64_t tiles, int64_t num_kb) {
+    int split = 1;
+    for (int i = 1; (1 << i) <= Umma2sCfg::kMaxSplit; ++i) {
+        const int s = 1 << i;
+        if (tiles <= h->stream_clusters[i] && num_kb >= 4 * s) split = s;
+    }
+    const int64_t cap = h->options[OPTIML_OPT_PAIR_SPLIT_MAX];
+    while (split > 1 && split > cap) split >>= 1;
+    return split;
+}
+
+// Whether the skinny kernel's schedule for this shape finishes every column tile in one CTA
+// (a single band: no partial tiles, no second pass).
+template <int MP, int SUB>
+bool skinny_single_band_cfg(optiml_handle_t h, int64_t N, int64_t K) {
+    using C = SkinnyCfg<MP, SUB>;
+    const int64_t max_slots = kPartialBytes / (C::kSlotFloats * sizeof(float));
+    const double unit_us = (double)(C::kBBytes + C::kABytes) / (kSkinnyCtaGBs * 1e3);
+    return make_skinny_plan(ceil_div64(N, C::BN), ceil_div64(K, C::BK), h->num_sms, max_slots, unit_us,
+                            kSkinnyAllGBs / kSkinnyCtaGBs).nbands == 1;
+}
+bool skinny_single_band(optiml_handle_t h, int64_t M, int64_t N, int64_t K) {
+    return M <= 64 ? skinny_single_band_cfg<64, 2>(h, N, K) : skinny_single_band_cfg<128, 2>(h, N, K);
 }
 
 // Shape-based choice.  fp32 goes to the FMA tiles.  bf16: M = 1 is a pure stream over B
@@ -184,16 +221,28 @@ int choose_variant(optiml_handle_t h, int64_t M, int64_t N, int64_t K, int dtype
     if (dtype == OPTIML_F32) {
         // fp32 has no tensor-core path: up to 4 rows stream over B (measured 1 x 8192 x 8192: 163 us
         // on the tiles, a fifth of that on the streaming kernel), everything else goes to the FMA tiles
-        if (M <= 4 && variant_supports(OPTIML_VARIANT_GEMV_SPLITK, M, N, K, dtype, al16)) return OPTIML_VARIANT_GEMV_SPLITK;
-        return variant_supports(OPTIML_VARIANT_F32_TILED, M, N, K, dtype, al16) ? OPTIML_VARIANT_F32_TILED
+        if (M <= 4 && variant_supports(h, OPTIML_VARIANT_GEMV_SPLITK, M, N, K, dtype, al16)) return OPTIML_VARIANT_GEMV_SPLITK;
+        return variant_supports(h, OPTIML_VARIANT_F32_TILED, M, N, K, dtype, al16) ? OPTIML_VARIANT_F32_TILED
                                                                                  : OPTIML_VARIANT_GENERIC;
     }
-    if (M == 1 && variant_supports(OPTIML_VARIANT_GEMV_SPLITK, M, N, K, dtype, al16)) return OPTIML_VARIANT_GEMV_SPLITK;
-    if (M <= 64 && variant_supports(OPTIML_VARIANT_SKINNY_UMMA, M, N, K, dtype, al16)) return OPTIML_VARIANT_SKINNY_UMMA;
+    if (M == 1 && variant_supports(h, OPTIML_VARIANT_GEMV_SPLITK, M, N, K, dtype, al16)) return OPTIML_VARIANT_GEMV_SPLITK;
+    const bool skinny_ok = variant_supports(h, OPTIML_VARIANT_SKINNY_UMMA, M, N, K, dtype, al16);
+    const bool stream_ok = variant_supports(h, OPTIML_VARIANT_UMMA_2CTA_STREAM, M, N, K, dtype, al16);
+    if (M <= 32 && skinny_ok) return OPTIML_VARIANT_SKINNY_UMMA;
+    if (M <= 128 && skinny_ok) {
+        // Between 33 and 128 rows the streaming kernel with N as the MMA M dimension wins where every
+        // column tile is finished by one CTA (measured 64 x 14336 x 4096: 21.5 us against 27.1 us for the
+        // cluster kernel; 128 rows: 26.4 against 28.6 us), and loses where its tiles are cut along K
+        // (64 x 8192 x 8192: 31.3 against 28.7 us; 128 rows: 46.7 against 29.9 us).
+        if (!stream_ok || skinny_single_band(h, M, N, K)) return OPTIML_VARIANT_SKINNY_UMMA;
+        return OPTIML_VARIANT_UMMA_2CTA_STREAM;
+    }
+    // fewer tiles than CTA pairs: the problem is a stream over B; one cluster per tile, K cut across its pairs
+    if (stream_ok) return OPTIML_VARIANT_UMMA_2CTA_STREAM;
     // above 64 rows a CTA pair shares one 256 x 256 tile (a third less operand traffic per flop); measured
     // at least as fast as the single-CTA kernel from M = 96 up, which stays as a forced variant
-    if (variant_supports(OPTIML_VARIANT_UMMA_2CTA, M, N, K, dtype, al16)) return OPTIML_VARIANT_UMMA_2CTA;
-    if (variant_supports(OPTIML_VARIANT_UMMA, M, N, K, dtype, al16)) return OPTIML_VARIANT_UMMA;
+    if (variant_supports(h, OPTIML_VARIANT_UMMA_2CTA, M, N, K, dtype, al16)) return OPTIML_VARIANT_UMMA_2CTA;
+    if (variant_supports(h, OPTIML_VARIANT_UMMA, M, N, K, dtype, al16)) return OPTIML_VARIANT_UMMA;
     return OPTIML_VARIANT_GENERIC;
 }
 
@@ -322,10 +371,9 @@ optiml_status_t launch_skinny_cfg(optiml_handle_t h, const void* A, const void* 
     // all CTAs together at about 7 TB/s (measured: 16 x 14336 x 16384 as 112 whole tiles 67 us = 7.0 TB/s,
     // as two balanced bands on 148 CTAs 76 us; 8 x 28672 x 4096 as one band on 148 CTAs 37.6 us, as two
     // bands 46.7 us; 16 x 8192 x 8192 as three bands 22.9 us, as 64 whole tiles 26.3 us)
-    constexpr double kCtaGBs = 110.0, kAllGBs = 7000.0;
-    const double unit_us = (double)(C::kBBytes + C::kABytes) / (kCtaGBs * 1e3);
+    const double unit_us = (double)(C::kBBytes + C::kABytes) / (kSkinnyCtaGBs * 1e3);
     const SkinnyPlan plan = make_skinny_plan(ceil_div64(N, C::BN), ceil_div64(K, C::BK), h->num_sms, max_slots, unit_us,
-                                             kAllGBs / kCtaGBs);
+                                             kSkinnyAllGBs / kSkinnyCtaGBs);
     if (h->log) fprintf(stderr, "[optiml] skinny plan: G=%d S=%d k_split=%d G1=%d k_mid=%d G2=%d bands=%d\n", plan.G, plan.S, plan.k_split, plan.G1, plan.k_mid, plan.G2, plan.nbands);
     SkinnyTune tune;
     const int64_t want = h->options[OPTIML_OPT_SKINNY_RING_STAGES];
@@ -401,7 +449,7 @@ optiml_status_t launch_umma2(optiml_handle_t h, const void* A, const void* B, co
     if (!get_map(h, &ma, A, (uint64_t)M, (uint64_t)K, 128, 64) || !get_map(h, &mb, B, (uint64_t)K, (uint64_t)N, 64, 64) ||
         !get_map(h, &my, Y, (uint64_t)M, (uint64_t)N, 32, 64))
         return OPTIML_ERR_CUDA;
-    const UmmaPlan plan = make_umma2_plan(M, N, K, h->num_sms);
+    const UmmaPlan plan = make_umma2_plan(M, N, K, h->num_sms, (int)h->options[OPTIML_OPT_PAIR_SPLIT_MAX]);
     if ((size_t)plan.rem_tiles * plan.split * C::BM * C::BN * sizeof(float) > kPartialBytes) return OPTIML_ERR_UNSUPPORTED;
     if (2 * plan.rem_tiles > kNumCounters) return OPTIML_ERR_UNSUPPORTED;
     const dim3 grid(2 * plan.grid);          // CTA pairs: the kernel is compiled with cluster dimensions (2, 1, 1)
@@ -428,6 +476,75 @@ optiml_status_t launch_umma2(optiml_handle_t h, const void* A, const void* B, co
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
 }
 
+// The streaming pair kernel: programmatic dependent launch plus a cluster of 2 * split CTAs.
+template <int ACT>
+cudaError_t launch_umma2s_act(dim3 grid, int cluster, cudaStream_t st, const CUtensorMap& ma, const CUtensorMap& mb,
+                              __nv_bfloat16* Y, const __nv_bfloat16* bias, int M, int N, int K,
+                              const Umma2sPlan& plan, int* status) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(Umma2sCfg::kThreads);
+    cfg.dynamicSmemBytes = Umma2sCfg::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)cluster;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, gemm_umma2s_kernel<ACT>, ma, mb, Y, bias, M, N, K, plan, status);
+}
+
+optiml_status_t launch_umma2s(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
+                              int K, int act, cudaStream_t st) {
+    using C = Umma2sCfg;
+    CUtensorMap ma, mb;
+    if (!get_map(h, &ma, A, (uint64_t)M, (uint64_t)K, 128, 64) || !get_map(h, &mb, B, (uint64_t)K, (uint64_t)N, 64, 64))
+        return OPTIML_ERR_CUDA;
+    Umma2sPlan plan;
+    plan.tiles_m = (int)ceil_div64(M, C::BM);
+    plan.tiles_n = (int)ceil_div64(N, C::BN);
+    plan.num_kb = (int)ceil_div64(K, C::BK);
+    const int64_t tiles = (int64_t)plan.tiles_m * plan.tiles_n;
+    plan.split = stream_split(h, tiles, plan.num_kb);
+    if (h->log) fprintf(stderr, "[optiml] streaming pair plan: tiles=%lld split=%d kb=%d\n", (long long)tiles, plan.split, plan.num_kb);
+    const int cluster = 2 * plan.split;
+    const dim3 grid((unsigned)(tiles * cluster));
+    const __nv_bfloat16* bi = (const __nv_bfloat16*)bias;
+    switch (act) {
+    case OPTIML_ACT_RELU: launch_umma2s_act<kActRelu>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
+    case OPTIML_ACT_GELU_TANH: launch_umma2s_act<kActGeluTanh>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
+    case OPTIML_ACT_SIGMOID: launch_umma2s_act<kActSigmoid>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
+    default: launch_umma2s_act<kActNone>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
+    }
+    h->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+// Clusters of `cluster` CTAs of the streaming pair kernel that can be resident at the same time.
+int query_stream_clusters(int cluster) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(cluster * 64));
+    cfg.blockDim = dim3(Umma2sCfg::kThreads);
+    cfg.dynamicSmemBytes = Umma2sCfg::kSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_umma2s_kernel<kActNone>, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    return n;
+}
+
 template <typename F>
 bool set_smem(F* fn, int bytes) {
     return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
@@ -452,6 +569,10 @@ bool configure_kernels() {
     ok &= set_smem(gemm_umma2_kernel<kActRelu>, Umma2Cfg::kSmemBytes);
     ok &= set_smem(gemm_umma2_kernel<kActGeluTanh>, Umma2Cfg::kSmemBytes);
     ok &= set_smem(gemm_umma2_kernel<kActSigmoid>, Umma2Cfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActNone>, Umma2sCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActRelu>, Umma2sCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActGeluTanh>, Umma2sCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActSigmoid>, Umma2sCfg::kSmemBytes);
     ok &= set_skinny(gemm_skinny_umma_kernel<16, 2>, SkinnyCfg<16, 2>::kSmemBytes);
     ok &= set_skinny(gemm_skinny_umma_kernel<16, 3>, SkinnyCfg<16, 3>::kSmemBytes);
     ok &= set_skinny(gemm_skinny_umma_kernel<32, 2>, SkinnyCfg<32, 2>::kSmemBytes);
@@ -554,6 +675,9 @@ optiml_status_t optiml_create(optiml_handle_t* out, int device) {
     ok = cudaMemset(h->counters, 0, kNumCounters * sizeof(unsigned int)) == cudaSuccess;
     ok = ok && cudaMemset(h->status, 0, sizeof(int)) == cudaSuccess;
     ok = ok && configure_kernels();
+    if (ok)
+        for (int i = 0; i < 2; ++i) h->stream_clusters[i] = query_stream_clusters(2 << i);
+    if (h->log) fprintf(stderr, "[optiml] resident clusters of the streaming pair kernel: %d of 2 CTAs, %d of 4 CTAs\n", h->stream_clusters[0], h->stream_clusters[1]);
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
@@ -588,7 +712,7 @@ optiml_status_t optiml_gemm_epilogue(optiml_handle_t h, const void* A, const voi
     if (all & (es - 1)) return OPTIML_ERR_ALIGNMENT;
     const bool al16 = aligned16(A) && aligned16(B) && aligned16(bias) && aligned16(Y);
     const int v = choose_variant(h, M, N, K, (int)dtype, al16);
-    if (!variant_supports(v, M, N, K, (int)dtype, al16)) return OPTIML_ERR_UNSUPPORTED;
+    if (!variant_supports(h, v, M, N, K, (int)dtype, al16)) return OPTIML_ERR_UNSUPPORTED;
     if (h->log)
         fprintf(stderr, "[optiml] M=%lld N=%lld K=%lld dtype=%d act=%d -> %s\n", (long long)M, (long long)N,
                 (long long)K, (int)dtype, (int)act, optiml_variant_name(v));
@@ -607,6 +731,8 @@ optiml_status_t optiml_gemm_epilogue(optiml_handle_t h, const void* A, const voi
         return launch_umma(h, A, B, bias, Y, m, n, k, (int)act, st);
     case OPTIML_VARIANT_UMMA_2CTA:
         return launch_umma2(h, A, B, bias, Y, m, n, k, (int)act, st);
+    case OPTIML_VARIANT_UMMA_2CTA_STREAM:
+        return launch_umma2s(h, A, B, bias, Y, m, n, k, (int)act, st);
     default:
         return dtype == OPTIML_F32 ? launch_generic<float>(h, A, B, bias, Y, m, n, k, (int)act, st)
                                    : launch_generic<__nv_bfloat16>(h, A, B, bias, Y, m, n, k, (int)act, st);
@@ -783,6 +909,7 @@ const char* optiml_variant_name(int variant) {
     case OPTIML_VARIANT_SKINNY_UMMA: return "skinny_streamk_tcgen05";
     case OPTIML_VARIANT_UMMA: return "persistent_tcgen05";
     case OPTIML_VARIANT_UMMA_2CTA: return "persistent_tcgen05_cta_pair";
+    case OPTIML_VARIANT_UMMA_2CTA_STREAM: return "cluster_splitk_tcgen05_cta_pair";
     default: return "unknown";
     }
 }

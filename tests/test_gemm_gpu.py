@@ -92,10 +92,37 @@ def test_umma_variant(handle, M, N, K, act, variant):
     parity(handle, synth.make_case("c4", M=M, N=N, K=K, act=act), variant)
 
 
+@pytest.mark.parametrize("M,N,K", [(256, 256, 64),        # one tile, one K block: no split possible
+                                   (200, 520, 1096),      # 3 tiles, ragged everywhere; up to 4 K slices
+                                   (100, 264, 2048),      # M <= 128: the second CTA of every pair has no rows
+                                   (130, 1288, 520),      # two rows in the second CTA
+                                   (512, 776, 1032),      # two tile rows
+                                   (65, 4096, 4096),      # 16 tiles: clusters of 8 where the device holds 16 of them
+                                   (256, 8192, 1024)])    # 32 tiles
+@pytest.mark.parametrize("act", [RELU, GELU])
+@pytest.mark.parametrize("split_max", [1, 2, 4])
+def test_streaming_pair_variant(handle, M, N, K, act, split_max):
+    handle.set_option(V.OPT_PAIR_SPLIT_MAX, split_max)
+    try:
+        parity(handle, synth.make_case("c4", M=M, N=N, K=K, act=act), V.VARIANT_UMMA_2CTA_STREAM)
+    finally:
+        handle.set_option(V.OPT_PAIR_SPLIT_MAX, 8)
+
+
+def test_streaming_pair_variant_refuses_more_tiles_than_clusters(handle):
+    handle.force_variant(V.VARIANT_UMMA_2CTA_STREAM)
+    c = synth.make_case("c4", M=2048, N=4096, K=64)          # 128 tiles
+    A, B = H.to_device(c.A, c.dtype, (c.M, c.K)), H.to_device(c.B, c.dtype, (c.K, c.N))
+    with pytest.raises(binding.OptimlError) as e:
+        handle.gemm_epilogue(A, B, None, c.act)
+    assert e.value.code == binding.ERR_UNSUPPORTED
+
+
 def test_null_bias_and_act_none(handle):
     for variant, name, shape in ((V.VARIANT_F32_TILED, "c1", (64, 64, 64)), (V.VARIANT_GEMV_SPLITK, "c2", (1, 512, 512)),
                                  (V.VARIANT_SKINNY_UMMA, "c3", (16, 512, 512)), (V.VARIANT_UMMA, "c4", (256, 512, 256)),
                                  (V.VARIANT_UMMA_2CTA, "c4", (256, 512, 256)),
+                                 (V.VARIANT_UMMA_2CTA_STREAM, "c4", (256, 512, 1024)),
                                  (V.VARIANT_GENERIC, "c4", (50, 60, 70))):
         c = synth.make_case(name, M=shape[0], N=shape[1], K=shape[2], act=NONE)
         c.bias = None
@@ -107,7 +134,8 @@ def test_null_bias_and_act_none(handle):
                                                 (V.VARIANT_GEMV_SPLITK, "c2", 1, 1032, 2048),
                                                 (V.VARIANT_SKINNY_UMMA, "c3", 16, 1160, 1096),
                                                 (V.VARIANT_UMMA, "c4", 300, 520, 200),
-                                                (V.VARIANT_UMMA_2CTA, "c4", 300, 520, 1096)])
+                                                (V.VARIANT_UMMA_2CTA, "c4", 300, 520, 1096),
+                                                (V.VARIANT_UMMA_2CTA_STREAM, "c4", 300, 520, 1096)])
 def test_sigmoid_epilogue(handle, variant, name, M, N, K):
     parity(handle, synth.make_case(name, M=M, N=N, K=K, act=synth.ACT_SIGMOID), variant)
 
@@ -120,7 +148,8 @@ def test_sigmoid_epilogue(handle, variant, name, M, N, K):
     (V.VARIANT_GEMV_SPLITK, F32, 1, 1028, 4096), (V.VARIANT_GEMV_SPLITK, F32, 3, 260, 1000),
     (V.VARIANT_GEMV_SPLITK, BF16, 4, 520, 1000), (V.VARIANT_SKINNY_UMMA, BF16, 16, 1160, 1096),
     (V.VARIANT_SKINNY_UMMA, BF16, 48, 648, 2048), (V.VARIANT_UMMA, BF16, 384, 776, 1024),
-    (V.VARIANT_UMMA_2CTA, BF16, 384, 776, 1024), (V.VARIANT_UMMA_2CTA, BF16, 1000, 520, 320)])
+    (V.VARIANT_UMMA_2CTA, BF16, 384, 776, 1024), (V.VARIANT_UMMA_2CTA, BF16, 1000, 520, 320),
+    (V.VARIANT_UMMA_2CTA_STREAM, BF16, 384, 776, 1024), (V.VARIANT_UMMA_2CTA_STREAM, BF16, 100, 2056, 4096)])
 @pytest.mark.parametrize("act", [NONE, RELU])
 def test_integer_inputs_are_bit_exact(handle, variant, dtype, M, N, K, act):
     c = synth.integer_case(M, N, K, dtype, act, seed=11)
@@ -218,8 +247,11 @@ def test_dispatcher_choices(handle):
     assert sel(16, 14336, 4096, BF16) == V.VARIANT_SKINNY_UMMA
     assert sel(4096, 4096, 4096, BF16) == V.VARIANT_UMMA_2CTA
     assert sel(8192, 8192, 16384, BF16) == V.VARIANT_UMMA_2CTA
-    assert sel(128, 4096, 4096, BF16) == V.VARIANT_UMMA_2CTA
-    assert sel(64, 4096, 4096, BF16) == V.VARIANT_SKINNY_UMMA and sel(2, 4096, 4096, BF16) == V.VARIANT_SKINNY_UMMA
+    assert sel(128, 4096, 4096, BF16) == V.VARIANT_UMMA_2CTA_STREAM     # 16 tiles for 74 CTA pairs
+    assert sel(256, 8192, 8192, BF16) == V.VARIANT_UMMA_2CTA_STREAM
+    assert sel(32, 4096, 4096, BF16) == V.VARIANT_SKINNY_UMMA and sel(2, 4096, 4096, BF16) == V.VARIANT_SKINNY_UMMA
+    assert sel(64, 14336, 4096, BF16) == V.VARIANT_SKINNY_UMMA          # every column tile whole in one CTA
+    assert sel(64, 8192, 8192, BF16) == V.VARIANT_UMMA_2CTA_STREAM      # the skinny schedule would cut tiles along K
     assert sel(4096, 4100, 4096, BF16) == V.VARIANT_GENERIC      # N % 8 != 0
     assert sel(0, 1, 1, BF16) == -1
 
