@@ -23,10 +23,19 @@ struct F32Cfg {
     static constexpr int kLdA = BM + 4;                    // padded, keeps float4 alignment
     static constexpr int kStage = kF32BK * kLdA + kF32BK * BN;   // floats per K-slice stage
     static constexpr int kSmemFloats = 2 * KS * kStage;
+    // A thread's TM rows (TN columns) are TM / 4 (TN / 4) groups of four, the groups spread evenly
+    // over the tile: neighbouring threads then read neighbouring float4s of a stage (no bank
+    // conflict), where one block of 8 consecutive columns per thread made every other thread of a
+    // quarter-warp hit the same banks.
+    static constexpr int kRowGroupStride = BM / (TM / 4), kColGroupStride = BN / (TN / 4);
+    // two CTAs per SM for the large tile (the compiler keeps it within 128 registers)
+    static constexpr int kMinCtas = (BM == 128 && BN == 128 && KS == 1) ? 2 : 1;
+    __host__ __device__ static constexpr int row_of(int ty, int i) { return (i / 4) * kRowGroupStride + ty * 4 + i % 4; }
+    __host__ __device__ static constexpr int col_of(int tx, int j) { return (j / 4) * kColGroupStride + tx * 4 + j % 4; }
 };
 
 template <int BM, int BN, int TM, int TN, int KS, int ACT>
-__global__ void __launch_bounds__(F32Cfg<BM, BN, TM, TN, KS>::kThreads)
+__global__ void __launch_bounds__(F32Cfg<BM, BN, TM, TN, KS>::kThreads, F32Cfg<BM, BN, TM, TN, KS>::kMinCtas)
 gemm_f32_tiled_kernel(const float* __restrict__ A, const float* __restrict__ B, const float* __restrict__ bias,
                       float* __restrict__ Y, int M, int N, int K) {
     using C = F32Cfg<BM, BN, TM, TN, KS>;
@@ -111,11 +120,12 @@ gemm_f32_tiled_kernel(const float* __restrict__ A, const float* __restrict__ B, 
         }
     };
 
-    float acc[TM][TN];
+    // accumulators as pairs of neighbouring columns: the operand form of the packed FMA below
+    float2 acc2[TM][TN / 2];
 #pragma unroll
     for (int i = 0; i < TM; ++i)
 #pragma unroll
-        for (int j = 0; j < TN; ++j) acc[i][j] = 0.0f;
+        for (int j = 0; j < TN / 2; ++j) acc2[i][j] = make_float2(0.0f, 0.0f);
 
     // Every K slice runs the same number of loop trips so the barriers line up; a slice
     // that has run out of steps loads zeros (its step index is past the end of K).
@@ -136,14 +146,19 @@ gemm_f32_tiled_kernel(const float* __restrict__ A, const float* __restrict__ B, 
 #pragma unroll
                 for (int i = 0; i < TM; i += 4)
                     *reinterpret_cast<float4*>(&av[i]) =
-                        *reinterpret_cast<const float4*>(a + kk * C::kLdA + ty * TM + i);
+                        *reinterpret_cast<const float4*>(a + kk * C::kLdA + C::row_of(ty, i));
 #pragma unroll
                 for (int j = 0; j < TN; j += 4)
-                    *reinterpret_cast<float4*>(&bv[j]) = *reinterpret_cast<const float4*>(b + kk * BN + tx * TN + j);
+                    *reinterpret_cast<float4*>(&bv[j]) = *reinterpret_cast<const float4*>(b + kk * BN + C::col_of(tx, j));
+                // packed FMAs (two fp32 lanes per instruction, each an ordinary round-to-nearest fp32
+                // FMA): half the issue slots of 64 scalar FMAs, which leaves room for the loads
 #pragma unroll
-                for (int i = 0; i < TM; ++i)
+                for (int i = 0; i < TM; ++i) {
+                    const float2 aa = make_float2(av[i], av[i]);
 #pragma unroll
-                    for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+                    for (int j = 0; j < TN / 2; ++j)
+                        acc2[i][j] = ptx::ffma2(aa, make_float2(bv[2 * j], bv[2 * j + 1]), acc2[i][j]);
+                }
             }
         }
         if (s + 1 < steps_per) {
@@ -152,6 +167,15 @@ gemm_f32_tiled_kernel(const float* __restrict__ A, const float* __restrict__ B, 
             buf ^= 1;
         }
     }
+
+    float acc[TM][TN];
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < TN / 2; ++j) {
+            acc[i][2 * j] = acc2[i][j].x;
+            acc[i][2 * j + 1] = acc2[i][j].y;
+        }
 
     if (KS > 1) {
         // Sum the K slices in slice order: slices 1..KS-1 park their tiles in shared memory
@@ -175,11 +199,11 @@ gemm_f32_tiled_kernel(const float* __restrict__ A, const float* __restrict__ B, 
 
 #pragma unroll
     for (int i = 0; i < TM; ++i) {
-        const int64_t m = m0 + ty * TM + i;
+        const int64_t m = m0 + C::row_of(ty, i);
         if (m >= M) continue;
 #pragma unroll
         for (int j = 0; j < TN; j += 4) {
-            const int64_t n = n0 + tx * TN + j;
+            const int64_t n = n0 + C::col_of(tx, j);
             if (n >= N) continue;      // N % 4 == 0: the float4 is wholly inside or outside
             float4 bv = bias ? *reinterpret_cast<const float4*>(bias + n) : make_float4(0, 0, 0, 0);
             float4 o;

@@ -20,6 +20,7 @@
 #include "kernel_generic.cuh"
 #include "kernel_mhsa.cuh"
 #include "kernel_reduce.cuh"
+#include "kernel_repack.cuh"
 #include "kernel_selftest.cuh"
 #include "kernel_skinny.cuh"
 #include "kernel_umma.cuh"
@@ -110,8 +111,10 @@ struct optiml_handle_s {
     encode_tiled_fn encode = nullptr;
     MapEntry maps[kMapCache];
     int next_map = 0;
-    void* stage[4] = {nullptr, nullptr, nullptr, nullptr};
+    void* stage[4] = {nullptr, nullptr, nullptr, nullptr};     // host entry point: A, B, bias, Y on the device
     size_t stage_bytes[4] = {0, 0, 0, 0};
+    void* pad[4] = {nullptr, nullptr, nullptr, nullptr};       // re-pitched copies of A, B, bias, Y (unaligned bf16 shapes)
+    size_t pad_bytes[4] = {0, 0, 0, 0};
     int64_t options[OPTIML_OPT_COUNT];
     int stream_clusters[2] = {0, 0};      // clusters of 2 and of 4 CTAs of the streaming pair kernel the device can hold at once
 };
@@ -622,6 +625,30 @@ bool mhsa_umma_supported(int64_t d_model, int64_t heads, int dtype, bool al16) {
     return dtype == OPTIML_BF16 && (dk == 64 || dk == 128) && al16 && heads <= 65535;
 }
 
+// Grow one of the handle's on-demand device buffers to `need` bytes.  Earlier work on the
+// stream may still use the old buffer, so the stream is synchronised before it is freed.
+optiml_status_t grow_buffer(void** buf, size_t* have, size_t need, cudaStream_t st) {
+    if (*have >= need) return OPTIML_OK;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return OPTIML_ERR_CUDA;
+    cudaFree(*buf);
+    *buf = nullptr;
+    *have = 0;
+    if (!dev_alloc(buf, need)) return OPTIML_ERR_ALLOC;   // the handle stays usable; this buffer is empty
+    *have = need;
+    return OPTIML_OK;
+}
+
+int64_t round_up8(int64_t x) { return (x + 7) / 8 * 8; }
+
+// bf16 problems whose N or K is not a multiple of 8 cannot be addressed by TMA in place.  Large
+// ones are worth two or three extra streaming passes: A (if K is ragged) and B (if N is ragged)
+// are copied into zero-padded buffers with 16-byte row pitches, the fast variant for the padded
+// shape runs into a padded Y, and the leading N columns are copied back.  (4096 x 4100 x 4096:
+// 5.6 ms on the predicated FMA kernel.)
+optiml_status_t gemm_repacked(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int64_t M,
+                              int64_t N, int64_t K, optiml_act_t act, void* stream);
+bool worth_repacking(int64_t M, int64_t N, int64_t K) { return M >= 16 && (double)M * (double)N * (double)K >= 134217728.0; }
+
 optiml_status_t check_args(optiml_handle_t h, const void* A, const void* B, const void* Y, int64_t M, int64_t N,
                            int64_t K, int dtype, int act) {
     if (!h || !A || !B || !Y) return OPTIML_ERR_INVALID_ARG;
@@ -696,6 +723,7 @@ optiml_status_t optiml_destroy(optiml_handle_t h) {
     cudaFree(h->counters);
     cudaFree(h->status);
     for (int i = 0; i < 4; ++i) cudaFree(h->stage[i]);
+    for (int i = 0; i < 4; ++i) cudaFree(h->pad[i]);
     cudaGetLastError();
     delete h;
     return OPTIML_OK;
@@ -711,6 +739,8 @@ optiml_status_t optiml_gemm_epilogue(optiml_handle_t h, const void* A, const voi
                           reinterpret_cast<uintptr_t>(bias) | reinterpret_cast<uintptr_t>(Y);
     if (all & (es - 1)) return OPTIML_ERR_ALIGNMENT;
     const bool al16 = aligned16(A) && aligned16(B) && aligned16(bias) && aligned16(Y);
+    if (dtype == OPTIML_BF16 && (N % 8 != 0 || K % 8 != 0) && al16 && h->forced == OPTIML_VARIANT_AUTO && worth_repacking(M, N, K))
+        return gemm_repacked(h, A, B, bias, Y, M, N, K, act, stream);
     const int v = choose_variant(h, M, N, K, (int)dtype, al16);
     if (!variant_supports(h, v, M, N, K, (int)dtype, al16)) return OPTIML_ERR_UNSUPPORTED;
     if (h->log)
@@ -739,6 +769,60 @@ optiml_status_t optiml_gemm_epilogue(optiml_handle_t h, const void* A, const voi
     }
 }
 
+}  // extern "C"
+
+namespace {
+
+optiml_status_t gemm_repacked(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int64_t M,
+                              int64_t N, int64_t K, optiml_act_t act, void* stream) {
+    DeviceGuard guard(h->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t Np = round_up8(N), Kp = round_up8(K);
+    const bool pad_a = Kp != K, pad_n = Np != N;
+    const size_t need[4] = {pad_a ? (size_t)M * Kp * 2 : 0, (size_t)Kp * Np * 2, pad_n && bias ? (size_t)Np * 2 : 0,
+                            pad_n ? (size_t)M * Np * 2 : 0};
+    for (int i = 0; i < 4; ++i) {
+        const optiml_status_t s = grow_buffer(&h->pad[i], &h->pad_bytes[i], need[i], st);
+        if (s != OPTIML_OK) return s;
+    }
+    auto blocks = [&](int64_t rows, int64_t cols_pad) {
+        const int64_t want = ceil_div64(rows * (cols_pad / 8), kRepackThreads);
+        const int64_t cap = (int64_t)h->num_sms * 16;
+        return dim3((unsigned)(want < cap ? (want < 1 ? 1 : want) : cap));
+    };
+    const void *a = A, *b = B, *bi = bias;
+    void* y = Y;
+    if (pad_a) {
+        pad_rows_kernel<<<blocks(M, Kp), kRepackThreads, 0, st>>>((const uint16_t*)A, (uint16_t*)h->pad[0], M, M, K, Kp);
+        a = h->pad[0];
+        h->launches += 1;
+    }
+    // B always moves: its row pitch changes with N, and with a ragged K it gains zero rows up to Kp
+    pad_rows_kernel<<<blocks(Kp, Np), kRepackThreads, 0, st>>>((const uint16_t*)B, (uint16_t*)h->pad[1], K, Kp, N, Np);
+    b = h->pad[1];
+    h->launches += 1;
+    if (pad_n) {
+        y = h->pad[3];
+        if (bias) {
+            pad_rows_kernel<<<blocks(1, Np), kRepackThreads, 0, st>>>((const uint16_t*)bias, (uint16_t*)h->pad[2], 1, 1, N, Np);
+            bi = h->pad[2];
+            h->launches += 1;
+        }
+    }
+    if (cudaGetLastError() != cudaSuccess) return OPTIML_ERR_CUDA;
+    const optiml_status_t s = optiml_gemm_epilogue(h, a, b, bi, y, M, Np, Kp, OPTIML_BF16, act, stream);
+    if (s != OPTIML_OK) return s;
+    if (pad_n) {
+        unpad_rows_kernel<<<blocks(M, Np), kRepackThreads, 0, st>>>((const uint16_t*)h->pad[3], (uint16_t*)Y, M, N, Np);
+        h->launches += 1;
+    }
+    return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
 optiml_status_t optiml_gemm_epilogue_host(optiml_handle_t h, const void* A_host, const void* B_host,
                                           const void* bias_host, void* Y_host, int64_t M, int64_t N, int64_t K,
                                           optiml_dtype_t dtype, optiml_act_t act, void* stream) {
@@ -749,13 +833,8 @@ optiml_status_t optiml_gemm_epilogue_host(optiml_handle_t h, const void* A_host,
     const size_t es = dtype == OPTIML_F32 ? 4 : 2;
     const size_t need[4] = {(size_t)M * K * es, (size_t)K * N * es, (size_t)N * es, (size_t)M * N * es};
     for (int i = 0; i < 4; ++i) {
-        if (h->stage_bytes[i] >= need[i]) continue;
-        if (cudaStreamSynchronize(st) != cudaSuccess) return OPTIML_ERR_CUDA;   // earlier work may still use it
-        cudaFree(h->stage[i]);
-        h->stage[i] = nullptr;
-        h->stage_bytes[i] = 0;
-        if (!dev_alloc(&h->stage[i], need[i])) return OPTIML_ERR_ALLOC;   // the handle stays usable; this buffer is empty
-        h->stage_bytes[i] = need[i];
+        const optiml_status_t g = grow_buffer(&h->stage[i], &h->stage_bytes[i], need[i], st);
+        if (g != OPTIML_OK) return g;
     }
     bool ok = cudaMemcpyAsync(h->stage[0], A_host, need[0], cudaMemcpyHostToDevice, st) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(h->stage[1], B_host, need[1], cudaMemcpyHostToDevice, st) == cudaSuccess;
