@@ -239,7 +239,9 @@ optiml_status_t optiml_reduce_f32(optiml_handle_t h, optiml_reduce_t kind, const
  * d_k <= 256, unaligned pointers and OPTIML_F32 run on a plain FMA kernel (fp32 throughout; bf16
  * rounded once at the store).  d_k > 256 returns OPTIML_ERR_UNSUPPORTED.  A forced
  * OPTIML_VARIANT_GENERIC (optiml_force_variant) selects the FMA kernel; any other forced variant
- * demands the tensor-core kernel and returns UNSUPPORTED where it cannot run.
+ * demands the tensor-core kernel and returns UNSUPPORTED where it cannot run; a forced
+ * OPTIML_VARIANT_UMMA_2CTA selects, at d_k = 128, the form in which a pair of CTAs shares every
+ * K and V block (same arithmetic, same tolerance).
  *
  * Enqueued on `stream`; INVALID_ARG / ALIGNMENT / UNSUPPORTED before anything is launched, CUDA if
  * the launch failed; a device-side time-out is reported by optiml_get_last_status.

@@ -19,6 +19,7 @@
 #include "kernel_gemv.cuh"
 #include "kernel_generic.cuh"
 #include "kernel_mhsa.cuh"
+#include "kernel_mhsa2.cuh"
 #include "kernel_reduce.cuh"
 #include "kernel_repack.cuh"
 #include "kernel_selftest.cuh"
@@ -589,6 +590,8 @@ bool configure_kernels() {
     cudaFuncAttributes fa;
     ok = ok && cudaFuncGetAttributes(&fa, mhsa_umma_kernel<64>) == cudaSuccess && fa.numRegs >= MhsaCfg<64>::kLaunchRegs;
     ok = ok && cudaFuncGetAttributes(&fa, mhsa_umma_kernel<128>) == cudaSuccess && fa.numRegs >= MhsaCfg<128>::kLaunchRegs;
+    ok = ok && set_smem(mhsa_umma2_kernel, Mhsa2Cfg::kSmemBytes);
+    ok = ok && cudaFuncGetAttributes(&fa, mhsa_umma2_kernel) == cudaSuccess && fa.numRegs >= Mhsa2Cfg::kLaunchRegs;
     return ok;
 }
 
@@ -604,6 +607,22 @@ optiml_status_t launch_mhsa_umma(optiml_handle_t h, const void* Q, const void* K
     const dim3 grid((unsigned)ceil_div64(N, C::kQTiles * C::BQ), (unsigned)heads);
     launch_pdl(mhsa_umma_kernel<DK>, grid, dim3(C::kThreads), C::kSmemBytes, st, mq, mk, mv, (__nv_bfloat16*)Y, N,
                d_model, scale_log2, h->status);
+    h->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+// d_k = 128 as a CTA pair: 512 query rows per cluster of two CTAs, each staging half of every K and V block
+optiml_status_t launch_mhsa_umma2(optiml_handle_t h, const void* Q, const void* K, const void* V, void* Y, int N,
+                                  int d_model, int heads, cudaStream_t st) {
+    using C = Mhsa2Cfg;
+    CUtensorMap mq, mk, mv;
+    if (!get_map(h, &mq, Q, (uint64_t)N, (uint64_t)d_model, 128, 64) || !get_map(h, &mk, K, (uint64_t)N, (uint64_t)d_model, 64, 64) ||
+        !get_map(h, &mv, V, (uint64_t)N, (uint64_t)d_model, 128, 64))
+        return OPTIML_ERR_CUDA;
+    const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)C::DK));
+    const dim3 grid((unsigned)(2 * ceil_div64(N, 2 * C::kQTiles * C::BQ)), (unsigned)heads);   // the kernel is compiled with cluster dimensions (2, 1, 1)
+    launch_pdl(mhsa_umma2_kernel, grid, dim3(C::kThreads), C::kSmemBytes, st, mq, mk, mv, (__nv_bfloat16*)Y, N, d_model,
+               scale_log2, h->status);
     h->launches += 1;
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
 }
@@ -932,10 +951,16 @@ optiml_status_t optiml_mhsa(optiml_handle_t h, const void* Q, const void* K, con
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (h->log)
         fprintf(stderr, "[optiml] mhsa N=%lld d_model=%lld heads=%lld dtype=%d -> %s\n", (long long)N, (long long)d_model,
-                (long long)heads, (int)dtype, want_fast ? "mhsa_tcgen05" : "mhsa_generic_fma");
-    if (want_fast)
-        return dk == 64 ? launch_mhsa_umma<64>(h, Q, K, V, Y, (int)N, (int)d_model, (int)heads, st)
-                        : launch_mhsa_umma<128>(h, Q, K, V, Y, (int)N, (int)d_model, (int)heads, st);
+                (long long)heads, (int)dtype,
+                !want_fast ? "mhsa_generic_fma" : (dk == 128 && h->forced == OPTIML_VARIANT_UMMA_2CTA ? "mhsa_tcgen05_cta_pair" : "mhsa_tcgen05"));
+    if (want_fast) {
+        if (dk == 64) return launch_mhsa_umma<64>(h, Q, K, V, Y, (int)N, (int)d_model, (int)heads, st);
+        // d_k = 128: the single-CTA kernel; the CTA-pair kernel only as the forced variant OPTIML_VARIANT_UMMA_2CTA
+        // (measured at N = 16384, 16 heads: 1776 us against 2029 us for the pair in short regions, 2061 against
+        // 2056 us back to back under the power cap)
+        if (h->forced != OPTIML_VARIANT_UMMA_2CTA) return launch_mhsa_umma<128>(h, Q, K, V, Y, (int)N, (int)d_model, (int)heads, st);
+        return launch_mhsa_umma2(h, Q, K, V, Y, (int)N, (int)d_model, (int)heads, st);
+    }
     return dtype == OPTIML_F32 ? launch_mhsa_generic<float>(h, Q, K, V, Y, (int)N, (int)d_model, (int)heads, st)
                                : launch_mhsa_generic<__nv_bfloat16>(h, Q, K, V, Y, (int)N, (int)d_model, (int)heads, st);
 }

@@ -63,6 +63,33 @@ def test_tensor_core_kernel_matches_oracle(handle, n, d_model, heads):
     check_bf16(y, mhsa_oracle.mhsa(q, k, v, n, d_model, heads), v)
 
 
+# d_k = 128 also has a CTA-pair kernel (each CTA stages half of every K and V block), a forced variant only
+PAIR_CASES = [(257, 128, 1), (512, 128, 1), (513, 256, 2), (640, 384, 3), (1000, 256, 2), (1537, 128, 1), (4096, 256, 2),
+              (2048, 2048, 16)]
+
+
+@pytest.mark.parametrize("n,d_model,heads", PAIR_CASES + [(100, 128, 1), (256, 256, 2)])
+def test_cta_pair_kernel_matches_oracle(handle, n, d_model, heads):
+    q, k, v = synth.mhsa_inputs(n, d_model, BF16, seed=n + heads)
+    handle.force_variant(binding.VARIANT_UMMA_2CTA)
+    try:
+        y = run(handle, q, k, v, n, d_model, heads, BF16)
+    finally:
+        handle.force_variant(binding.VARIANT_AUTO)
+    check_bf16(y, mhsa_oracle.mhsa(q, k, v, n, d_model, heads), v)
+
+
+def test_cta_pair_kernel_with_late_maxima(handle):
+    n, d_model, heads = 1500, 256, 2
+    q, k, v = synth.mhsa_inputs(n, d_model, BF16, seed=7, q_gain=3.0, key_growth=3.0)
+    handle.force_variant(binding.VARIANT_UMMA_2CTA)
+    try:
+        y = run(handle, q, k, v, n, d_model, heads, BF16)
+    finally:
+        handle.force_variant(binding.VARIANT_AUTO)
+    check_bf16(y, mhsa_oracle.mhsa(q, k, v, n, d_model, heads), v)
+
+
 @pytest.mark.parametrize("d_model,heads", [(128, 2), (256, 2)])
 @pytest.mark.parametrize("q_gain,key_growth", [(4.0, 0.0), (1.0, 6.0), (3.0, 3.0), (16.0, 0.0)])
 def test_sharp_and_late_maxima(handle, d_model, heads, q_gain, key_growth):
