@@ -461,6 +461,20 @@ def measure(handle, name, case, bound, args, sampler, device, peaks, peak_src, c
     return res
 
 
+def isolated_floor_us(handle, device, sampler):
+    """What the isolated-call protocol measures for a kernel that does next to nothing (a 4-element
+    sum through the same C ABI): launch latency plus the two event records, the part of every
+    `single_call_us` figure that is not the kernel's own work."""
+    x = torch.ones(4, dtype=torch.float32, device=device)
+    out = torch.empty(1, dtype=torch.float32, device=device)
+    stream = torch.cuda.current_stream(device)
+    timer = Timer(lambda i: handle.reduce_f32(0, x, None, out=out, stream=stream), stream, device, sampler)
+    timer.warm(10)
+    iso = timer.isolated(SINGLE_CALLS)
+    return {"median": statistics.median(iso), "min": min(iso), "calls": len(iso),
+            "what": "isolated call of a 4-element sum: launch latency + event records"}
+
+
 def shape_entry(r):
     c, pc = r["case"], r["per_call_us"]
     e = {"workload": r["name"], "M": c.M, "N": c.N, "K": c.K, "variant": r["variant"],
@@ -794,6 +808,7 @@ def main():
             "per_shape": per_shape, "reductions": reductions, "attention": attention, "extra_shapes": extras}
     if "single_call_us" in main_res:
         line["single_call_us"] = main_res["single_call_us"]
+        line["single_call_floor_us"] = isolated_floor_us(handle, device, sampler)
     sampler.stop()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(case, unit)

@@ -832,7 +832,7 @@ optiml_status_t gemm_repacked(optiml_handle_t h, const void* A, const void* B, c
     const optiml_status_t s = optiml_gemm_epilogue(h, a, b, bi, y, M, Np, Kp, OPTIML_BF16, act, stream);
     if (s != OPTIML_OK) return s;
     if (pad_n) {
-        unpad_rows_kernel<<<blocks(M, Np), kRepackThreads, 0, st>>>((const uint16_t*)h->pad[3], (uint16_t*)Y, M, N, Np);
+        unpad_rows_kernel<<<blocks(M, Np), kRepackThreads, 0, st>>>((const uint16_t*)h->pad[3], (uint16_t*)Y, M, N, Np);   // Y is 16-byte aligned here
         h->launches += 1;
     }
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
