@@ -55,7 +55,7 @@ struct MhsaCfg {
     // (With 48 registers the MMA lanes of the d_k = 128 instantiation spilled two values that they
     // re-read every key block; 56 is what the pool leaves beside 2 x 128 x 224.)
     static constexpr int kThreads = 384;
-    static constexpr int kLaunchRegs = 168, kControlRegs = DK == 64 ? 48 : 56, kSoftmaxRegs = 224;
+    static constexpr int kLaunchRegs = 168, kControlRegs = 56, kSoftmaxRegs = 224;
     static_assert(128 * kControlRegs + 256 * kSoftmaxRegs <= kThreads * kLaunchRegs, "register shares exceed the launch's pool");
     static constexpr int kTmemCols = 512;                // S0, S1: 2 x 128; O0, O1: 2 x DK; P0, P1: 2 x 64
     static constexpr int kColS = 0, kColO = 256;
