@@ -71,9 +71,10 @@ struct SkinnyCfg {
     // on 16 x 14336 x 4096, one lane needed 0.9 us per 192-row stage, which capped a CTA at
     // 53 GB/s.  With two lanes each issues every other 16-row step of K into an accumulator of
     // its own (the epilogue adds the two, always in the same order).  The second set of
-    // accumulators halves the column tiles a sweep can hold (kAcc); at MP = 128 the MMAs are
-    // long enough (N = 128: 64 cycles on the pipe) for one lane.
-    static constexpr int kIssuers = MP <= 64 ? 2 : 1;
+    // accumulators halves the column tiles a sweep can hold (kAcc).  At MP = 128 an MMA takes 64
+    // cycles on the pipe, about what one lane needs to issue it; two lanes still gain 2-3 %
+    // (128 x 14336 x 4096: 26.3 -> 25.6 us), so every configuration has two.
+    static constexpr int kIssuers = 2;
     static constexpr int kThreads = 192 + 32 * (kIssuers - 1); // warp 6: the second issuing lane
     static constexpr int kAccFit = 256 / (MP * kIssuers);
     static constexpr int kAcc = kAccFit < 8 ? kAccFit : 8;     // column tiles per sweep
