@@ -182,7 +182,11 @@ gemm_umma2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             for (int wi = 0; ok && umma2_work_item(plan, pair, wi, w); ++wi) {
                 const int tm = w.tm, tn = w.tn;
                 if (sh->abort) { ok = false; break; }
-                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+                // whole tiles walk K forwards and backwards in turn: the end of the panels a wave has just
+                // streamed is what L2 still holds when the next tiles start (same order in the MMA lane)
+                const bool rev = w.rem_idx < 0 && (wi & 1);
+                for (int kbi = w.kb0; kbi < w.kb1; ++kbi, ++it) {
+                    const int kb = rev ? w.kb1 - 1 - (kbi - w.kb0) : kbi;
                     if ((site = 1, !ptx::mbar_wait(&sh->empty[s], ph ^ 1))) { ok = false; break; }
                     uint8_t* a_dst = ring + s * C::kStageBytes;
                     uint8_t* b_dst = a_dst + C::kABytes;
@@ -238,7 +242,7 @@ gemm_umma2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 if (sh->abort || (site = 2, !ptx::mbar_wait(&sh->tmem_empty[a], aph ^ 1))) { ok = false; break; }
                 ptx::tcgen05_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + a * C::BN;
-                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
+                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {     // kb counts the K blocks in the order the producer sends them
                     // (the abort flag is looked at once per tile, above: every wait is bounded anyway)
                     if ((site = 4, !ptx::mbar_wait(&sh->full[s], ph))) { ok = false; break; }
                     ptx::tcgen05_fence_after_sync();

@@ -221,6 +221,23 @@ gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
         const int chunk_cols = C::BN / S;                   // columns this CTA finishes: 256 or 128
         const float4* recv = reinterpret_cast<const float4*>(ring + C::kRecvOffset) + row;
+        const int64_t row0 = (int64_t)tm * C::BM + hc * 128 + q * 32;       // first row of this warp
+        const int64_t col0 = (int64_t)tn * C::BN + band * chunk_cols;       // first column of this CTA's chunk
+        const int nblk = chunk_cols / 128;                                  // 64-column blocks per warp: 2 or 1
+
+        // The bias of this warp's columns is fetched now, while the main loop runs: at the end nothing
+        // but the accumulator stands between the last MMA and the stores.
+        uint4 bias_w[2][2][4];                              // [block][32-column group][8 columns]
+#pragma unroll
+        for (int bi = 0; bi < 2; ++bi)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    const int64_t n = col0 + ((colhalf * nblk + bi) * 2 + hh) * 32 + v * 8;
+                    bias_w[bi][hh][v] = (bias && bi < nblk && n < N) ? *reinterpret_cast<const uint4*>(bias + n)   // N % 8 == 0
+                                                                     : make_uint4(0, 0, 0, 0);
+                }
 
         bool ok = (kb1 > kb0) && !sh->abort && ptx::mbar_wait(&sh->tmem_full, 0);
         ok = __all_sync(0xffffffffu, ok);
@@ -257,6 +274,16 @@ gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 else
                     site = 8;                           // reported below; the partner's wait for the share runs out too
             }
+        }
+
+        // this warp's own share of its first 64-column block leaves tensor memory while the partner's
+        // share is still on its way
+        uint32_t racc[2][32];
+        if (ok && rows_live) {
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) ptx::tmem_ld_32x32(t_lane + band * chunk_cols + (colhalf * nblk * 2 + hh) * 32, racc[hh]);
+        }
+        if (S > 1) {
             if (ok && rows_live && !ptx::mbar_wait(&sh->recv_full, 0)) {
                 ok = false;
                 site = 9;
@@ -266,18 +293,20 @@ gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
 
         if (ok && rows_live) {
             // ---- sum in band order, bias + activation, one rounding, store
-            const int64_t row0 = (int64_t)tm * C::BM + hc * 128 + q * 32;       // first row of this warp
-            const int64_t col0 = (int64_t)tn * C::BN + band * chunk_cols;       // first column of this CTA's chunk
-            const int nblk = chunk_cols / 128;                                  // 64-column blocks per warp: 2 or 1
-            for (int bi = 0; bi < nblk; ++bi) {
+#pragma unroll
+            for (int bi = 0; bi < 2; ++bi) {
+                if (bi >= nblk) break;
                 const int blk = colhalf * nblk + bi;                            // 64-column block within the chunk
+                if (bi > 0) {
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) ptx::tmem_ld_32x32(t_lane + band * chunk_cols + (blk * 2 + hh) * 32, racc[hh]);
+                }
+                ptx::tmem_ld_wait();
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
                     const int g = blk * 2 + hh;             // 32-column group within the chunk
                     float x[32];
-                    uint32_t r[32];
-                    ptx::tmem_ld_32x32(t_lane + band * chunk_cols + g * 32, r);
-                    ptx::tmem_ld_wait();
+                    const uint32_t (&r)[32] = racc[hh];
                     if (S > 1) {
                         float4 t[8];
 #pragma unroll
@@ -304,8 +333,7 @@ gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
                         const int64_t n = col0 + g * 32 + v * 8;
-                        uint4 bw = make_uint4(0, 0, 0, 0);
-                        if (bias && n < N) bw = *reinterpret_cast<const uint4*>(bias + n);    // N % 8 == 0
+                        const uint4 bw = bias_w[bi][hh][v];
                         const uint32_t bwv[4] = {bw.x, bw.y, bw.z, bw.w};
                         uint32_t o[4];
 #pragma unroll
