@@ -97,6 +97,9 @@ def main():
     ap.add_argument("--n", type=int, default=1 << 26, help="vector length for --reduce")
     ap.add_argument("--mhsa", choices=sorted(synth.MHSA_WORKLOADS), help="run multi-head self-attention instead")
     ap.add_argument("--heads", type=int, help="with --mhsa: override the head count (and --N, --K = d_model)")
+    ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE",
+                    help="optiml_set_option before the run, e.g. gemv_prefetch_rows=48, skinny_stage_rows=128, "
+                         "skinny_ring_stages=3, skinny_prefetch_early=2, skinny_late_trigger=0, pair_split_max=1")
     a = ap.parse_args()
     if a.reduce:
         return run_reduce(a)
@@ -107,6 +110,9 @@ def main():
     h = binding.Handle(0)
     if a.variant != "auto":
         h.force_variant(int(a.variant))
+    for item in a.option:
+        name, value = item.split("=")
+        h.set_option(getattr(binding, "OPT_" + name.upper()), int(value))
     tdt = torch.float32 if c.dtype == synth.F32 else torch.bfloat16
     A0, B0, b0 = _dev(c.A, c.dtype, (c.M, c.K)), _dev(c.B, c.dtype, (c.K, c.N)), _dev(c.bias, c.dtype, (c.N,))
     sets = [(A0, B0, b0, torch.empty((c.M, c.N), dtype=tdt, device="cuda"))]
