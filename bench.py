@@ -237,13 +237,18 @@ class Timer:
             torch.cuda.synchronize(self.device)
         return e0.elapsed_time(e1), t0, t1
 
-    def isolated(self, calls):
+    def isolated(self, calls, gate=None):
         """One pair of events around every call, the stream synchronised between calls: no call
-        overlaps the drain of the one before -> list of microseconds."""
+        overlaps the drain of the one before -> list of microseconds.  With `gate` (a callable that
+        enqueues a short busy kernel on the stream) the event records and the call are enqueued while
+        the GPU is still busy with the gate, so the time between the events holds no host latency:
+        what remains is the call alone, from an idle, drained GPU."""
         out = []
         for _ in range(calls):
             torch.cuda.synchronize(self.device)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            if gate is not None:
+                gate()
             e0.record(self.stream)
             self.step(self.i)
             self.i += 1
@@ -273,6 +278,27 @@ class Timer:
             win = sm.window(t2 + 0.05, time.perf_counter())
             how = "same load continued after the timed region (region shorter than the sampling period)"
         return summarise_clocks(win, sm.max_mhz, how)
+
+
+_GATE = {}
+
+
+def make_gate(device):
+    """A callable that enqueues a busy kernel of about 60 us on the current stream (the library's
+    bounded-wait self-test on a handle of its own, whose status word nobody else reads)."""
+    from paper_2602_12305_b200 import binding
+    key = str(device)
+    if key not in _GATE:
+        _GATE[key] = binding.Handle(device.index if device.index is not None else 0)
+    gh = _GATE[key]
+    return lambda: gh.selftest_timeout(120000)
+
+
+def close_gates():
+    for gh in _GATE.values():
+        gh.get_last_status()          # clears the recorded time-outs
+        gh.destroy()
+    _GATE.clear()
 
 
 def protocol(timer, min_launches, est_ms):
@@ -408,9 +434,12 @@ def measure_once(handle, name, case, bound, args, sampler, device, peaks, peak_s
     if bound == "tensor" and not quick:
         out["sustained"] = sustained(timer, stats["median"])
     if bound != "tensor" and not quick:
-        iso = timer.isolated(SINGLE_CALLS)
+        iso = timer.isolated(SINGLE_CALLS, gate=make_gate(device))
+        host = timer.isolated(SINGLE_CALLS)
         out["single_call_us"] = {"median": statistics.median(iso), "min": min(iso), "calls": len(iso),
-                                 "how": "one call between two events, stream synchronised before each call"}
+                                 "how": "one call between two events on a drained GPU; a short busy kernel ahead of the "
+                                        "first event hides the host's enqueue latency",
+                                 "with_host_latency_median": statistics.median(host)}
     out["launches"] = handle.launch_count() - launches0
     del sets, timer
     torch.cuda.empty_cache()
@@ -470,9 +499,11 @@ def isolated_floor_us(handle, device, sampler):
     stream = torch.cuda.current_stream(device)
     timer = Timer(lambda i: handle.reduce_f32(0, x, None, out=out, stream=stream), stream, device, sampler)
     timer.warm(10)
-    iso = timer.isolated(SINGLE_CALLS)
+    iso = timer.isolated(SINGLE_CALLS, gate=make_gate(device))
+    host = timer.isolated(SINGLE_CALLS)
     return {"median": statistics.median(iso), "min": min(iso), "calls": len(iso),
-            "what": "isolated call of a 4-element sum: launch latency + event records"}
+            "with_host_latency_median": statistics.median(host),
+            "what": "isolated call of a 4-element sum: kernel start-up + event records"}
 
 
 def shape_entry(r):
@@ -533,7 +564,7 @@ def measure_reductions(handle, device, sampler, peaks, peak_src, quick):
                             "frac": gbs / peaks["hbm_gbs"], "traffic": TRAFFIC.get(name), "algorithmic_bytes": nbytes,
                             "peak_source": f"of {peak_src}: copy bandwidth"}}
         if not quick:
-            iso = timer.isolated(SINGLE_CALLS)
+            iso = timer.isolated(SINGLE_CALLS, gate=make_gate(device))
             row["single_call_us"] = {"median": statistics.median(iso), "min": min(iso), "calls": len(iso),
                                      "gbs": nbytes / 1e3 / statistics.median(iso),
                                      "frac": nbytes / 1e3 / statistics.median(iso) / peaks["hbm_gbs"]}
@@ -837,6 +868,7 @@ def main():
             row += ["sustained", round(s["us_per_call"], 1), round(s["frac"], 3), s["launches"]]
         summary.append(row)
     line["summary"] = summary
+    close_gates()
     handle.destroy()
     replicas.barrier()
     if rank == 0:

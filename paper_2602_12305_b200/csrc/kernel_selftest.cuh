@@ -19,8 +19,7 @@ __global__ void __launch_bounds__(32, 1) selftest_timeout_kernel(long long limit
         ptx::fence_mbar_init();
     }
     __syncwarp();
-    ptx::griddep_wait();
-    ptx::griddep_launch_dependents();
+    ptx::griddep_wait();        // (no early trigger: whatever follows in the stream starts when this kernel is over)
     if (threadIdx.x == 0) {
         // phase 0 never completes: there is no arrival and no expected byte count
         if (!ptx::mbar_wait_limit(&bar, 0, limit_cycles)) report_timeout(status, kSelftestWaitSite);
