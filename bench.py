@@ -826,7 +826,7 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": region_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32" if case.dtype == synth.F32 else "bf16", "data": "synthetic",
-            "config": workload_config(case, name, main_res["variant"]),
+            "config": workload_config(case, name, None), "variant": main_res["variant"],
             "tflops": case.flops / 1e12 * world / (region_ms / args.steps / 1e3),
             "gbs": case.algorithmic_bytes / 1e9 * world / (region_ms / args.steps / 1e3),
             "roofline": head_rl, "clocks": main_res["contract_clocks"],
