@@ -100,8 +100,8 @@ optiml_status_t optiml_destroy(optiml_handle_t h);
  * has run; the library keeps no reference after that.  Pointers must be aligned
  * to the element size; the fast variants also need 16-byte aligned pointers and
  * N, K multiples of 8 (bf16) or 4 (fp32) -- other shapes run on the generic
- * variant, never on the CPU.  One exception: a large bf16 problem (M >= 16, M N K >= 2^27)
- * with 16-byte aligned pointers whose N or K is not a multiple of 8 is copied into
+ * variant, never on the CPU.  One exception: a large problem (M >= 16, M N K >= 2^27)
+ * with 16-byte aligned pointers whose N or K is not a multiple of 8 (bf16) or 4 (fp32) is copied into
  * zero-padded buffers with 16-byte row pitches (A if K is ragged, B always, Y on the way
  * back if N is ragged) and runs on the fast variants; those buffers belong to the handle
  * and grow on demand, which synchronises `stream` and allocates on the first such call and

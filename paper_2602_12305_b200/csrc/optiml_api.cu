@@ -657,15 +657,14 @@ optiml_status_t grow_buffer(void** buf, size_t* have, size_t need, cudaStream_t 
     return OPTIML_OK;
 }
 
-int64_t round_up8(int64_t x) { return (x + 7) / 8 * 8; }
-
-// bf16 problems whose N or K is not a multiple of 8 cannot be addressed by TMA in place.  Large
-// ones are worth two or three extra streaming passes: A (if K is ragged) and B (if N is ragged)
-// are copied into zero-padded buffers with 16-byte row pitches, the fast variant for the padded
-// shape runs into a padded Y, and the leading N columns are copied back.  (4096 x 4100 x 4096:
-// 5.6 ms on the predicated FMA kernel.)
+// Problems whose N or K is not a multiple of 16 bytes' worth of elements (8 bf16, 4 fp32) cannot be
+// addressed by TMA, nor by the 128-bit loads of the fp32 tiles, in place.  Large ones are worth two or
+// three extra streaming passes: A (if K is ragged) and B are copied into zero-padded buffers with
+// 16-byte row pitches, the fast variant for the padded shape runs into a padded Y (if N is ragged),
+// and the leading N columns are copied back.  (bf16 4096 x 4100 x 4096: 5.6 ms on the predicated FMA
+// kernel, 0.14 ms this way.)
 optiml_status_t gemm_repacked(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int64_t M,
-                              int64_t N, int64_t K, optiml_act_t act, void* stream);
+                              int64_t N, int64_t K, optiml_dtype_t dtype, optiml_act_t act, void* stream);
 bool worth_repacking(int64_t M, int64_t N, int64_t K) { return M >= 16 && (double)M * (double)N * (double)K >= 134217728.0; }
 
 optiml_status_t check_args(optiml_handle_t h, const void* A, const void* B, const void* Y, int64_t M, int64_t N,
@@ -758,8 +757,9 @@ optiml_status_t optiml_gemm_epilogue(optiml_handle_t h, const void* A, const voi
                           reinterpret_cast<uintptr_t>(bias) | reinterpret_cast<uintptr_t>(Y);
     if (all & (es - 1)) return OPTIML_ERR_ALIGNMENT;
     const bool al16 = aligned16(A) && aligned16(B) && aligned16(bias) && aligned16(Y);
-    if (dtype == OPTIML_BF16 && (N % 8 != 0 || K % 8 != 0) && al16 && h->forced == OPTIML_VARIANT_AUTO && worth_repacking(M, N, K))
-        return gemm_repacked(h, A, B, bias, Y, M, N, K, act, stream);
+    const int64_t vec = dtype == OPTIML_F32 ? 4 : 8;       // elements per 16 bytes
+    if ((N % vec != 0 || K % vec != 0) && al16 && h->forced == OPTIML_VARIANT_AUTO && worth_repacking(M, N, K))
+        return gemm_repacked(h, A, B, bias, Y, M, N, K, dtype, act, stream);
     const int v = choose_variant(h, M, N, K, (int)dtype, al16);
     if (!variant_supports(h, v, M, N, K, (int)dtype, al16)) return OPTIML_ERR_UNSUPPORTED;
     if (h->log)
@@ -792,50 +792,59 @@ optiml_status_t optiml_gemm_epilogue(optiml_handle_t h, const void* A, const voi
 
 namespace {
 
-optiml_status_t gemm_repacked(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int64_t M,
-                              int64_t N, int64_t K, optiml_act_t act, void* stream) {
+template <typename E>
+optiml_status_t gemm_repacked_t(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int64_t M,
+                                int64_t N, int64_t K, optiml_dtype_t dtype, optiml_act_t act, void* stream) {
+    constexpr int64_t V = RepackVec<E>::V;
     DeviceGuard guard(h->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int64_t Np = round_up8(N), Kp = round_up8(K);
+    const int64_t Np = (N + V - 1) / V * V, Kp = (K + V - 1) / V * V;
     const bool pad_a = Kp != K, pad_n = Np != N;
-    const size_t need[4] = {pad_a ? (size_t)M * Kp * 2 : 0, (size_t)Kp * Np * 2, pad_n && bias ? (size_t)Np * 2 : 0,
-                            pad_n ? (size_t)M * Np * 2 : 0};
+    const size_t es = sizeof(E);
+    const size_t need[4] = {pad_a ? (size_t)M * Kp * es : 0, (size_t)Kp * Np * es, pad_n && bias ? (size_t)Np * es : 0,
+                            pad_n ? (size_t)M * Np * es : 0};
     for (int i = 0; i < 4; ++i) {
         const optiml_status_t s = grow_buffer(&h->pad[i], &h->pad_bytes[i], need[i], st);
         if (s != OPTIML_OK) return s;
     }
     auto blocks = [&](int64_t rows, int64_t cols_pad) {
-        const int64_t want = ceil_div64(rows * (cols_pad / 8), kRepackThreads);
+        const int64_t want = ceil_div64(rows * (cols_pad / V), kRepackThreads);
         const int64_t cap = (int64_t)h->num_sms * 16;
         return dim3((unsigned)(want < cap ? (want < 1 ? 1 : want) : cap));
     };
     const void *a = A, *b = B, *bi = bias;
     void* y = Y;
     if (pad_a) {
-        pad_rows_kernel<<<blocks(M, Kp), kRepackThreads, 0, st>>>((const uint16_t*)A, (uint16_t*)h->pad[0], M, M, K, Kp);
+        pad_rows_kernel<E><<<blocks(M, Kp), kRepackThreads, 0, st>>>((const E*)A, (E*)h->pad[0], M, M, K, Kp);
         a = h->pad[0];
         h->launches += 1;
     }
     // B always moves: its row pitch changes with N, and with a ragged K it gains zero rows up to Kp
-    pad_rows_kernel<<<blocks(Kp, Np), kRepackThreads, 0, st>>>((const uint16_t*)B, (uint16_t*)h->pad[1], K, Kp, N, Np);
+    pad_rows_kernel<E><<<blocks(Kp, Np), kRepackThreads, 0, st>>>((const E*)B, (E*)h->pad[1], K, Kp, N, Np);
     b = h->pad[1];
     h->launches += 1;
     if (pad_n) {
         y = h->pad[3];
         if (bias) {
-            pad_rows_kernel<<<blocks(1, Np), kRepackThreads, 0, st>>>((const uint16_t*)bias, (uint16_t*)h->pad[2], 1, 1, N, Np);
+            pad_rows_kernel<E><<<blocks(1, Np), kRepackThreads, 0, st>>>((const E*)bias, (E*)h->pad[2], 1, 1, N, Np);
             bi = h->pad[2];
             h->launches += 1;
         }
     }
     if (cudaGetLastError() != cudaSuccess) return OPTIML_ERR_CUDA;
-    const optiml_status_t s = optiml_gemm_epilogue(h, a, b, bi, y, M, Np, Kp, OPTIML_BF16, act, stream);
+    const optiml_status_t s = optiml_gemm_epilogue(h, a, b, bi, y, M, Np, Kp, dtype, act, stream);
     if (s != OPTIML_OK) return s;
     if (pad_n) {
-        unpad_rows_kernel<<<blocks(M, Np), kRepackThreads, 0, st>>>((const uint16_t*)h->pad[3], (uint16_t*)Y, M, N, Np);   // Y is 16-byte aligned here
+        unpad_rows_kernel<E><<<blocks(M, Np), kRepackThreads, 0, st>>>((const E*)h->pad[3], (E*)Y, M, N, Np);   // Y is 16-byte aligned here
         h->launches += 1;
     }
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+optiml_status_t gemm_repacked(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int64_t M,
+                              int64_t N, int64_t K, optiml_dtype_t dtype, optiml_act_t act, void* stream) {
+    return dtype == OPTIML_F32 ? gemm_repacked_t<uint32_t>(h, A, B, bias, Y, M, N, K, dtype, act, stream)
+                               : gemm_repacked_t<uint16_t>(h, A, B, bias, Y, M, N, K, dtype, act, stream);
 }
 
 }  // namespace

@@ -272,6 +272,19 @@ def test_large_unaligned_bf16_shapes_take_the_fast_variants_through_padded_copie
     assert np.array_equal(bits, bits2)
 
 
+@pytest.mark.parametrize("M,N,K", [(520, 518, 520), (520, 520, 517), (300, 1030, 1001), (1100, 1026, 260)])
+def test_large_unaligned_fp32_shapes_take_the_tile_kernel_through_padded_copies(handle, M, N, K):
+    c = synth.make_case("c1", M=M, N=N, K=K, act=GELU)
+    before = handle.launch_count()
+    bits = parity(handle, c)
+    assert handle.launch_count() - before >= 3
+    bits2, _ = H.run_case(handle, c)
+    assert np.array_equal(bits, bits2)
+    ci = synth.integer_case(M, N, K, F32, RELU, seed=3)
+    bi, _ = H.run_case(handle, ci)
+    H.check_bit_exact(bi, H.oracle_full(ci), F32, f"unaligned fp32 {M}x{N}x{K} through padded copies")
+
+
 def test_padded_copies_keep_integer_cases_exact(handle):
     c = synth.integer_case(300, 1030, 1001, BF16, RELU, seed=5)
     bits, _ = H.run_case(handle, c)
