@@ -255,7 +255,9 @@ optiml_status_t optiml_mhsa(optiml_handle_t h, const void* Q, const void* K, con
 optiml_status_t optiml_force_variant(optiml_handle_t h, optiml_variant_t v);
 
 /* Variant the dispatcher would run for this problem (honours a forced variant;
- * pointers are assumed 16-byte aligned), or -1 on bad arguments. */
+ * pointers are assumed 16-byte aligned), or -1 on bad arguments.  A large unaligned
+ * shape that optiml_gemm_epilogue re-pitches is reported as OPTIML_VARIANT_GENERIC here;
+ * ask with N and K rounded up to the vector width for the variant its padded copy runs on. */
 int optiml_select_variant(optiml_handle_t h, int64_t M, int64_t N, int64_t K, optiml_dtype_t dtype);
 
 /*
