@@ -452,10 +452,12 @@ def measure(handle, name, case, bound, args, sampler, device, peaks, peak_src, c
     from paper_2602_12305_b200 import binding
     res = measure_once(handle, name, case, bound, args, sampler, device, peaks, peak_src, contract_steps, quick)
     remeasured, timeouts = False, 0
-    if clocks_rejected(res["clocks"]) or (contract_steps and clocks_rejected(res["contract_clocks"])):
+    # (every rank takes the same decision: the contract region holds barriers)
+    if replicas.any_rank(clocks_rejected(res["clocks"]) or bool(contract_steps and clocks_rejected(res["contract_clocks"])),
+                         device):
         res = measure_once(handle, name, case, bound, args, sampler, device, peaks, peak_src, contract_steps, quick)
         remeasured = True
-    if handle.get_last_status() != binding.OK:
+    if replicas.any_rank(handle.get_last_status() != binding.OK, device):
         # a bounded on-device wait gave up: the timing is void; measure once more and say so
         timeouts = 1
         res = measure_once(handle, name, case, bound, args, sampler, device, peaks, peak_src, contract_steps, quick)

@@ -49,6 +49,16 @@ def aggregate(elapsed_ms: float, units: float, device: torch.device | str = "cpu
     return float(t.item()), float(u.item())
 
 
+def any_rank(flag: bool, device: torch.device | str = "cpu") -> bool:
+    """True on every rank if `flag` is true on any rank.  Decisions that change how many barriers a
+    rank goes through (measuring a workload again) must be taken alike by all ranks."""
+    if not dist.is_initialized():
+        return bool(flag)
+    t = torch.tensor([1 if flag else 0], dtype=torch.int32, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return bool(t.item())
+
+
 def shutdown():
     if dist.is_initialized():
         dist.destroy_process_group()

@@ -22,6 +22,7 @@ def _worker(rank, world, port, out):
     assert (r, w) == (rank, world)
     replicas.barrier()
     ms, units = replicas.aggregate(10.0 + 5.0 * rank, 3.0 + rank)     # rank 1 is slower and did more
+    assert replicas.any_rank(rank == 1) is True and replicas.any_rank(False) is False
     out.put((rank, ms, units))
     replicas.barrier()
     replicas.shutdown()
@@ -49,3 +50,4 @@ def test_single_process_is_a_pass_through(monkeypatch):
     assert replicas.init("gloo") == (0, 1)
     replicas.barrier()
     assert replicas.aggregate(2.5, 4.0) == (2.5, 4.0)
+    assert replicas.any_rank(True) is True and replicas.any_rank(False) is False
