@@ -237,6 +237,27 @@ def test_c4_c5_sampled(handle, name):
     assert np.array_equal(bits, bits2)
 
 
+@pytest.mark.parametrize("M,N,K", [(256, 8192, 8192),      # 32 tiles, two CTA pairs per tile: the exchange between the pairs
+                                   (128, 8192, 8192),      # the same with an empty second CTA in every pair
+                                   (256, 14336, 4096),     # 56 tiles, one pair per tile
+                                   (512, 8192, 8192)])     # two rows of tiles
+def test_crossover_shapes_of_the_cluster_kernel_on_sampled_outputs(handle, M, N, K):
+    """The shapes of the dispatcher's crossover table at full size, as the benchmark launches them."""
+    c = synth.make_case("c4", M=M, N=N, K=K)
+    assert handle.select_variant(M, N, K, c.dtype) == V.VARIANT_UMMA_2CTA_STREAM
+    bits, y = H.run_case(handle, c)
+    rows = sample_indices(M, 128, 96, 1)
+    cols = sample_indices(N, 256, 320, 2)
+    ref = oracle.gemm_epilogue_sampled(c.A, c.B, c.bias, M, N, K, c.dtype, c.act, rows, cols)
+    H.check_tolerance(y[np.ix_(rows, cols)], ref, c.dtype, f"{M}x{N}x{K} sampled {len(rows)}x{len(cols)}")
+    frows = np.array([0, M // 2 + 3, M - 1])
+    ref_r = oracle.gemm_epilogue_sampled(c.A, c.B, c.bias, M, N, K, c.dtype, c.act, frows, np.arange(N))
+    H.check_tolerance(y[frows], ref_r, c.dtype, "full rows")
+    assert np.isfinite(y).all()
+    bits2, _ = H.run_case(handle, c)
+    assert np.array_equal(bits, bits2)
+
+
 # ---------------------------------------------------------------- dispatcher, metamorphic relations, edge cases
 
 def test_dispatcher_choices(handle):
