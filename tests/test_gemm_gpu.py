@@ -258,6 +258,26 @@ def test_crossover_shapes_of_the_cluster_kernel_on_sampled_outputs(handle, M, N,
     assert np.array_equal(bits, bits2)
 
 
+def _random_shapes(seed, count):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(count):
+        dtype = BF16 if rng.random() < 0.7 else F32
+        M = int(rng.choice([1, 2, 7, 16, 33, 64, 65, 100, 128, 129, 200, 256, 300, 513, 700]))
+        N = int(rng.integers(1, 40)) * int(rng.choice([8, 8, 64, 72, 128])) + int(rng.choice([0, 0, 0, 1, 2, 4]))
+        K = int(rng.integers(1, 40)) * int(rng.choice([8, 16, 64, 96])) + int(rng.choice([0, 0, 0, 1, 3, 4]))
+        act = int(rng.choice([NONE, RELU, GELU, synth.ACT_SIGMOID]))
+        out.append((dtype, M, N, K, act))
+    return out
+
+
+@pytest.mark.parametrize("dtype,M,N,K,act", _random_shapes(2024, 60))
+def test_random_shapes_through_the_dispatcher(handle, dtype, M, N, K, act):
+    """Whatever the dispatcher picks for a shape (aligned or not, any regime), the result matches the oracle."""
+    c = synth.make_case("c1" if dtype == F32 else "c4", M=M, N=N, K=K, act=act)
+    parity(handle, c)
+
+
 # ---------------------------------------------------------------- dispatcher, metamorphic relations, edge cases
 
 def test_dispatcher_choices(handle):
@@ -280,6 +300,7 @@ def test_dispatcher_choices(handle):
 @pytest.mark.parametrize("M,N,K", [(520, 516, 520),        # N ragged
                                    (520, 520, 516),        # K ragged
                                    (300, 1030, 1001),      # both ragged, odd K
+                                   (300, 1031, 1000),      # odd N: rows of B and Y start on 2-byte boundaries only
                                    (64, 2052, 1100),       # lands on the skinny kernel
                                    (1100, 1028, 260)])
 @pytest.mark.parametrize("act", [RELU, GELU])
@@ -293,7 +314,7 @@ def test_large_unaligned_bf16_shapes_take_the_fast_variants_through_padded_copie
     assert np.array_equal(bits, bits2)
 
 
-@pytest.mark.parametrize("M,N,K", [(520, 518, 520), (520, 520, 517), (300, 1030, 1001), (1100, 1026, 260)])
+@pytest.mark.parametrize("M,N,K", [(520, 518, 520), (520, 520, 517), (300, 1030, 1001), (300, 1031, 1003), (1100, 1026, 260)])
 def test_large_unaligned_fp32_shapes_take_the_tile_kernel_through_padded_copies(handle, M, N, K):
     c = synth.make_case("c1", M=M, N=N, K=K, act=GELU)
     before = handle.launch_count()
