@@ -337,13 +337,13 @@ mhsa_umma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     m_used = mx;
                 }
 #pragma unroll 1
-                for (int c = 0; c < DK / 32; ++c) {
-                    uint32_t o[32];
-                    ptx::tmem_ld_32x32(o_addr + c * 32, o);
+                for (int c = 0; c < DK / 8; ++c) {          // 8 columns at a time: the whole row of scores is live here
+                    uint32_t o[8];
+                    ptx::tmem_ld_32x8(o_addr + c * 8, o);
                     ptx::tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                    ptx::tmem_st_32x32(o_addr + c * 32, o);
+                    for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    ptx::tmem_st_32x8(o_addr + c * 8, o);
                 }
                 ptx::tmem_st_wait();
             }

@@ -48,7 +48,7 @@ struct Mhsa2Cfg {
     static constexpr int kPBytes = 2 * kChunkBytes;      // 128 x 128 bf16 probabilities
     static constexpr int kKSlots = 3, kVSlots = 3;
     static constexpr int kThreads = 384;
-    static constexpr int kLaunchRegs = 168, kControlRegs = 56, kSoftmaxRegs = 224;
+    static constexpr int kLaunchRegs = 168, kControlRegs = 88, kSoftmaxRegs = 208;   // (56 / 224 spilled two values here)
     static_assert(128 * kControlRegs + 256 * kSoftmaxRegs <= kThreads * kLaunchRegs, "register shares exceed the launch's pool");
     static constexpr int kTmemCols = 512;                // S0, S1: 2 x 128; O0, O1: 2 x 128
     static constexpr int kColS = 0, kColO = 256;
@@ -313,13 +313,13 @@ mhsa_umma2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     m_used = mx;
                 }
 #pragma unroll 1
-                for (int c = 0; c < DK / 32; ++c) {
-                    uint32_t o[32];
-                    ptx::tmem_ld_32x32(o_addr + c * 32, o);
+                for (int c = 0; c < DK / 8; ++c) {          // 8 columns at a time: the whole row of scores is live here
+                    uint32_t o[8];
+                    ptx::tmem_ld_32x8(o_addr + c * 8, o);
                     ptx::tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                    ptx::tmem_st_32x32(o_addr + c * 32, o);
+                    for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    ptx::tmem_st_32x8(o_addr + c * 8, o);
                 }
                 ptx::tmem_st_wait();
             }
