@@ -83,22 +83,30 @@ gemm_f32_tiled_kernel(const float* __restrict__ A, const float* __restrict__ B, 
     auto Bs = [&](int buf) { return stage0 + buf * C::kStage + kF32BK * C::kLdA; };
 
     float4 ra[kAVec], rb[kBVec];
+    // What does not change from step to step is computed once: the thread's first source pointers at
+    // k = 0 (its further float4s lie a fixed number of rows below) and whether its rows of A / columns of
+    // B lie inside the matrices (one bit each).
+    constexpr int kARowStep = C::kGroup / (kF32BK / 4);     // rows of A between a thread's consecutive float4s
+    constexpr int kBRowStep = C::kGroup / (BN / 4);         // rows of B between a thread's consecutive float4s
+    static_assert(C::kGroup % (kF32BK / 4) == 0 && C::kGroup % (BN / 4) == 0, "a thread keeps its column within a stage");
+    const int a_r0 = g / (kF32BK / 4), a_c = (g % (kF32BK / 4)) * 4;
+    const int b_r0 = g / (BN / 4), b_c = (g % (BN / 4)) * 4;
+    const float* a_src = A + (m0 + a_r0) * K + a_c;
+    const float* b_src = B + (int64_t)b_r0 * N + n0 + b_c;
+    const bool b_live = n0 + b_c < N;
+    unsigned a_live = 0;
+#pragma unroll
+    for (int i = 0; i < kAVec; ++i) a_live |= (m0 + a_r0 + i * kARowStep < M ? 1u : 0u) << i;
     auto load_global = [&](int step) {
-        const int64_t k0 = (int64_t)step * kF32BK;
+        const int k0 = step * kF32BK;
 #pragma unroll
-        for (int i = 0; i < kAVec; ++i) {
-            const int e = g + i * C::kGroup;           // float4 index in the BM x (BK/4) tile
-            const int r = e / (kF32BK / 4), c4 = e % (kF32BK / 4);
-            const int64_t m = m0 + r, k = k0 + c4 * 4;
-            ra[i] = (m < M && k < K) ? *reinterpret_cast<const float4*>(A + m * K + k) : make_float4(0, 0, 0, 0);
-        }
+        for (int i = 0; i < kAVec; ++i)
+            ra[i] = ((a_live >> i) & 1u) && k0 + a_c < K
+                        ? *reinterpret_cast<const float4*>(a_src + (int64_t)(i * kARowStep) * K + k0) : make_float4(0, 0, 0, 0);
 #pragma unroll
-        for (int i = 0; i < kBVec; ++i) {
-            const int e = g + i * C::kGroup;           // float4 index in the BK x (BN/4) tile
-            const int r = e / (BN / 4), c4 = e % (BN / 4);
-            const int64_t k = k0 + r, n = n0 + c4 * 4;
-            rb[i] = (k < K && n < N) ? *reinterpret_cast<const float4*>(B + k * N + n) : make_float4(0, 0, 0, 0);
-        }
+        for (int i = 0; i < kBVec; ++i)
+            rb[i] = b_live && k0 + b_r0 + i * kBRowStep < K
+                        ? *reinterpret_cast<const float4*>(b_src + (int64_t)(k0 + i * kBRowStep) * N) : make_float4(0, 0, 0, 0);
     };
     auto store_shared = [&](int buf) {
         float* a = As(buf);
