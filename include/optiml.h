@@ -284,7 +284,9 @@ typedef enum {
                                              0 = as soon as the kernel starts                                       */
     OPTIML_OPT_PAIR_SPLIT_MAX = 5,        /* CTA-pair GEMMs: most K slices a tile is cut into (persistent form: tiles of
                                              the last, partial round, up to 8; streaming form: 1 or 2)          */
-    OPTIML_OPT_COUNT = 6
+    OPTIML_OPT_PAIR_HALF_HEIGHT = 6,      /* streaming CTA-pair form, M <= 128: 1 = 128-row tiles, 64 rows per CTA
+                                             (default), 0 = 256-row tiles as for larger M                            */
+    OPTIML_OPT_COUNT = 7
 } optiml_option_t;
 optiml_status_t optiml_set_option(optiml_handle_t h, optiml_option_t opt, int64_t value);
 int64_t optiml_get_option(optiml_handle_t h, optiml_option_t opt);

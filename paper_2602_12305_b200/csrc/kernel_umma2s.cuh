@@ -37,24 +37,40 @@
 
 namespace optiml {
 
-struct Umma2sCfg {
-    static constexpr int BM = 256, BN = 256, BK = 64, kStages = 6;
-    static constexpr int kABytes = 128 * 64 * 2;             // this CTA's 128 rows x 64 k of A
+// HM ("half-height"): the pair's tile is 128 rows high, 64 per CTA (tcgen05.mma.cta_group::2 with
+// M = 128), for M <= 128.  With 256-row tiles such a problem leaves the second CTA of every pair
+// multiplying zero rows while the first pulls 128 rows of A and 128 columns of B through its SM's
+// port; here each CTA pulls 64 rows and 128 columns, a quarter less per SM, and both do useful
+// work.  The accumulator of a CTA then sits in tensor memory as lanes [0, 64) = its 64 rows x
+// columns [0, 128) of the tile and lanes [64, 128) = the same rows x columns [128, 256):
+// 128 tensor-memory columns in all.
+template <bool HM>
+struct Umma2sCfgT {
+    static constexpr int BM = HM ? 128 : 256, BN = 256, BK = 64, kStages = HM ? 8 : 6;
+    static constexpr int kRowsPerCta = BM / 2;
+    static constexpr int kABytes = kRowsPerCta * 64 * 2;     // this CTA's rows x 64 k of A
     static constexpr int kBChunkBytes = 64 * 64 * 2;         // 64 k x 64 columns
     static constexpr int kBBytes = 2 * kBChunkBytes;         // 64 k x this CTA's 128 columns of B
-    static constexpr int kStageBytes = kABytes + kBBytes;    // 32 KiB
+    static constexpr int kStageBytes = kABytes + kBBytes;    // 32 KiB (24 KiB)
     static constexpr int kEpiWarps = 8;
     static constexpr int kThreads = 64 + 32 * kEpiWarps;
-    static constexpr int kTmemCols = 256;
-    // After the main loop the ring is reused: 64 KiB receive the partner's share (128 rows x 128
-    // columns of fp32), 64 KiB hold the share on its way to the partner.
-    static constexpr int kShareBytes = 128 * 128 * 4;
+    static constexpr int kTmemCols = HM ? 128 : 256;
+    // After the main loop the ring is reused: one share (the half of this CTA's accumulator that
+    // the partner finishes: 128 rows x 128 columns of fp32, or 64 x 128) is received, one is held
+    // on its way to the partner.
+    static constexpr int kShareBytes = kRowsPerCta * 128 * 4;
     static constexpr int kRecvOffset = 0, kSendOffset = kShareBytes;
     static constexpr int kRingBytes = kStages * kStageBytes;
+    static_assert(kStageBytes % 1024 == 0, "swizzle atoms start on 1024-byte boundaries");
     static_assert(kSendOffset + kShareBytes <= kRingBytes, "ring reuse");
     static constexpr int kSmemBytes = kRingBytes + 256 + 1024;
     static constexpr int kMaxSplit = 2;                      // cluster of 4 CTAs
 };
+using Umma2sCfg = Umma2sCfgT<false>;
+using Umma2sHalfCfg = Umma2sCfgT<true>;
+static_assert(Umma2sCfg::kSmemBytes == Umma2sHalfCfg::kSmemBytes && Umma2sCfg::kThreads == Umma2sHalfCfg::kThreads,
+              "both forms launch alike (the resident-cluster counts are queried once)");
+constexpr int kUmma2sMaxStages = 8;
 
 struct Umma2sPlan {
     int tiles_m, tiles_n, num_kb;
@@ -62,8 +78,8 @@ struct Umma2sPlan {
 };
 
 struct Umma2sShared {
-    uint64_t full[Umma2sCfg::kStages];     // used in the pair's leader: bytes of both CTAs land here
-    uint64_t empty[Umma2sCfg::kStages];    // per CTA, signalled by the leader's commit
+    uint64_t full[kUmma2sMaxStages];       // used in the pair's leader: bytes of both CTAs land here
+    uint64_t empty[kUmma2sMaxStages];      // per CTA, signalled by the leader's commit
     uint64_t tmem_full;                    // per CTA, signalled by the leader's commit
     uint64_t drain;
     uint64_t partner_idle;                 // the partner's main loop is over: its ring may be written
@@ -71,6 +87,7 @@ struct Umma2sShared {
     uint32_t tmem_base;
     volatile int abort;
 };
+static_assert(sizeof(Umma2sShared) <= 256, "barrier block");
 
 __device__ __forceinline__ void umma2s_epi_bar_sync() { asm volatile("bar.sync 4, 256;" ::: "memory"); }
 
@@ -93,13 +110,13 @@ __device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster, const
                  : "memory");
 }
 
-template <int ACT>
-__global__ void __launch_bounds__(Umma2sCfg::kThreads, 1)
+template <int ACT, bool HM>
+__global__ void __launch_bounds__(Umma2sCfgT<HM>::kThreads, 1)
 gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                    __nv_bfloat16* __restrict__ Y,
                    const __nv_bfloat16* __restrict__ bias, int M, int N, int K, const __grid_constant__ Umma2sPlan plan,
                    int* __restrict__ status) {
-    using C = Umma2sCfg;
+    using C = Umma2sCfgT<HM>;
     extern __shared__ uint8_t smem_raw[];
     Umma2sShared* sh = reinterpret_cast<Umma2sShared*>(smem_raw);
     const uint32_t ring_base = (ptx::smem_u32(smem_raw) + 256 + 1023) & ~1023u;
@@ -156,7 +173,7 @@ gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 uint8_t* b_dst = a_dst + C::kABytes;
                 const uint32_t full_leader = full_leader0 + 8u * s;
                 ptx::mbar_arrive_expect_tx_cluster(full_leader, C::kStageBytes);
-                ptx::tma_load_2d_2cta(a_dst, &map_a, full_leader, kb * C::BK, tm * C::BM + hc * 128);
+                ptx::tma_load_2d_2cta(a_dst, &map_a, full_leader, kb * C::BK, tm * C::BM + hc * C::kRowsPerCta);
 #pragma unroll
                 for (int j = 0; j < 2; ++j)
                     ptx::tma_load_2d_2cta(b_dst + j * C::kBChunkBytes, &map_b, full_leader, tn * C::BN + hc * 128 + j * 64,
@@ -211,7 +228,7 @@ gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             ptx::umma_commit_2cta_local(&sh->drain);
             ptx::mbar_wait(&sh->drain, 0);
         }
-    } else {
+    } else if constexpr (!HM) {
         // ------------------------------------------------------------ epilogue warps
         const int ew = warp - 2;                            // 0..7 among the epilogue warps
         const int q = warp & 3;                             // tensor-memory lane quarter this warp may read
@@ -344,6 +361,122 @@ gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                         }
                         if (m < M && n < N) *reinterpret_cast<uint4*>(Y + m * N + n) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
+                }
+            }
+        }
+        if (!ok && lane == 0 && kb1 > kb0) {
+            report_timeout(status, site);
+            sh->abort = 1;
+        }
+        if (site == 8) report_timeout(status, 8);
+    } else {
+        // ------------------------------------------------------------ epilogue warps, 64 rows per CTA
+        // Tensor-memory lane L holds row L % 64 of this CTA; its 128 columns are columns
+        // [128 (L / 64), 128 (L / 64) + 128) of the tile.  With S = 2 band b finishes tensor-memory
+        // columns [64 b, 64 b + 64) of every lane and hands the other 64 to its partner (a 32 KiB
+        // share); with S = 1 a CTA finishes all 128.  Of the two warps on a lane quarter each takes
+        // half of those columns.
+        const int ew = warp - 2, q = warp & 3, ch = ew >> 2;
+        const int L = q * 32 + lane;
+        const bool rows_live = (int64_t)tm * C::BM + hc * C::kRowsPerCta < M;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
+        const int ngroups = S == 1 ? 2 : 1;                                  // 32-column groups this warp finishes
+        const int keep0 = S == 1 ? 64 * ch : 64 * band + 32 * ch;            // its first tensor-memory column
+        const int64_t m = (int64_t)tm * C::BM + hc * C::kRowsPerCta + (L & 63);
+        const int64_t n0 = (int64_t)tn * C::BN + (q >> 1) * 128 + keep0;     // first column of Y of this thread
+        const float4* recv = reinterpret_cast<const float4*>(ring + C::kRecvOffset) + L;
+
+        uint4 bias_w[2][4];                                 // fetched while the main loop runs
+#pragma unroll
+        for (int g = 0; g < 2; ++g)
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                const int64_t n = n0 + g * 32 + v * 8;
+                bias_w[g][v] = (bias && g < ngroups && n < N) ? *reinterpret_cast<const uint4*>(bias + n)   // N % 8 == 0
+                                                              : make_uint4(0, 0, 0, 0);
+            }
+
+        bool ok = (kb1 > kb0) && !sh->abort && ptx::mbar_wait(&sh->tmem_full, 0);
+        ok = __all_sync(0xffffffffu, ok);
+        int site = 5;
+        ptx::tcgen05_fence_after_sync();
+
+        if (S > 1) {
+            if (ok && threadIdx.x == 64) ptx::mbar_arrive_cluster(ptx::mapa_shared(ptx::smem_u32(&sh->partner_idle), partner));
+            if (ok && rows_live) {
+                // float4 index (column / 4) * 128 + lane: a warp writes (and later reads) 512 contiguous bytes
+                float4* send = reinterpret_cast<float4*>(ring + C::kSendOffset) + L;
+                uint32_t r[32];
+                ptx::tmem_ld_32x32(t_lane + 64 * (band ^ 1) + 32 * ch, r);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int v = 0; v < 8; ++v)
+                    send[(ch * 8 + v) * 128] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                           __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                ptx::fence_proxy_async_smem();
+            }
+            umma2s_epi_bar_sync();
+            if (threadIdx.x == 64 && ok && rows_live) {
+                if (ptx::mbar_wait(&sh->partner_idle, 0))
+                    bulk_copy_to_cluster(ptx::mapa_shared(ring_base + C::kRecvOffset, partner), ring + C::kSendOffset,
+                                         C::kShareBytes, ptx::mapa_shared(ptx::smem_u32(&sh->recv_full), partner));
+                else
+                    site = 8;
+            }
+        }
+
+        uint32_t racc[2][32];
+        if (ok && rows_live) {
+#pragma unroll
+            for (int g = 0; g < 2; ++g)
+                if (g < ngroups) ptx::tmem_ld_32x32(t_lane + keep0 + g * 32, racc[g]);
+        }
+        if (S > 1) {
+            if (ok && rows_live && !ptx::mbar_wait(&sh->recv_full, 0)) {
+                ok = false;
+                site = 9;
+            }
+            ok = __all_sync(0xffffffffu, ok);
+        }
+
+        if (ok && rows_live) {
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+                if (g >= ngroups) break;
+                float x[32];
+                const uint32_t (&r)[32] = racc[g];
+                if (S > 1) {
+                    float4 t[8];
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) t[v] = recv[(ch * 8 + v) * 128];
+                    // band 0 holds the first half of K: its share comes first in the sum
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        const float p[4] = {t[v].x, t[v].y, t[v].z, t[v].w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float mine = __uint_as_float(r[4 * v + i]);
+                            x[4 * v + i] = band == 0 ? mine + p[i] : p[i] + mine;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) x[i] = __uint_as_float(r[i]);
+                }
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    const int64_t n = n0 + g * 32 + v * 8;
+                    const uint4 bw = bias_w[g][v];
+                    const uint32_t bwv[4] = {bw.x, bw.y, bw.z, bw.w};
+                    uint32_t o[4];
+#pragma unroll
+                    for (int p = 0; p < 4; ++p) {
+                        const float y0 = epilogue<ACT, true>(x[v * 8 + 2 * p], bf16lo_to_f32(bwv[p]));
+                        const float y1 = epilogue<ACT, true>(x[v * 8 + 2 * p + 1], bf16hi_to_f32(bwv[p]));
+                        o[p] = pack_bf16x2(y0, y1);
+                    }
+                    if (m < M && n < N) *reinterpret_cast<uint4*>(Y + m * N + n) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
             }
         }

@@ -47,6 +47,7 @@ constexpr int64_t kOptionDefaults[OPTIML_OPT_COUNT] = {
     /* SKINNY_PREFETCH_EARLY */ 4,
     /* SKINNY_LATE_TRIGGER   */ 1,
     /* PAIR_SPLIT_MAX        */ 8,
+    /* PAIR_HALF_HEIGHT      */ 1,
 };
 
 // Streaming rates the skinny kernel's schedule is costed with (see launch_skinny_cfg).
@@ -234,11 +235,12 @@ int choose_variant(optiml_handle_t h, int64_t M, int64_t N, int64_t K, int dtype
     const bool stream_ok = variant_supports(h, OPTIML_VARIANT_UMMA_2CTA_STREAM, M, N, K, dtype, al16);
     if (M <= 32 && skinny_ok) return OPTIML_VARIANT_SKINNY_UMMA;
     if (M <= 128 && skinny_ok) {
-        // Between 33 and 128 rows the streaming kernel with N as the MMA M dimension wins where every
-        // column tile is finished by one CTA (measured 64 x 14336 x 4096: 21.5 us against 27.1 us for the
-        // cluster kernel; 128 rows: 26.4 against 28.6 us), and loses where its tiles are cut along K
-        // (64 x 8192 x 8192: 31.3 against 28.7 us; 128 rows: 46.7 against 29.9 us).
-        if (!stream_ok || skinny_single_band(h, M, N, K)) return OPTIML_VARIANT_SKINNY_UMMA;
+        // Between 33 and 128 rows the streaming kernel with N as the MMA M dimension wins up to 64 rows where
+        // every column tile is finished by one CTA (measured 64 x 14336 x 4096: 21.9 us against 23.0 us for
+        // the cluster kernel with 64 rows per CTA), and loses above (128 rows: 25.7 against 23.7 us) and
+        // wherever its tiles are cut along K (64 x 8192 x 8192: 31.3 against 25.5 us; 128 rows: 41.4
+        // against 25.6 us).
+        if (!stream_ok || (M <= 64 && skinny_single_band(h, M, N, K))) return OPTIML_VARIANT_SKINNY_UMMA;
         return OPTIML_VARIANT_UMMA_2CTA_STREAM;
     }
     // fewer tiles than CTA pairs: the problem is a stream over B; one cluster per tile, K cut across its pairs
@@ -481,7 +483,7 @@ optiml_status_t launch_umma2(optiml_handle_t h, const void* A, const void* B, co
 }
 
 // The streaming pair kernel: programmatic dependent launch plus a cluster of 2 * split CTAs.
-template <int ACT>
+template <int ACT, bool HM>
 cudaError_t launch_umma2s_act(dim3 grid, int cluster, cudaStream_t st, const CUtensorMap& ma, const CUtensorMap& mb,
                               __nv_bfloat16* Y, const __nv_bfloat16* bias, int M, int N, int K,
                               const Umma2sPlan& plan, int* status) {
@@ -499,14 +501,18 @@ cudaError_t launch_umma2s_act(dim3 grid, int cluster, cudaStream_t st, const CUt
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, gemm_umma2s_kernel<ACT>, ma, mb, Y, bias, M, N, K, plan, status);
+    return cudaLaunchKernelEx(&cfg, gemm_umma2s_kernel<ACT, HM>, ma, mb, Y, bias, M, N, K, plan, status);
 }
 
-optiml_status_t launch_umma2s(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
-                              int K, int act, cudaStream_t st) {
-    using C = Umma2sCfg;
+// Up to 128 rows a pair shares a 128-row tile (64 rows per CTA); above, a 256-row tile.
+bool stream_half_height(optiml_handle_t h, int64_t M) { return M <= Umma2sHalfCfg::BM && h->options[OPTIML_OPT_PAIR_HALF_HEIGHT] != 0; }
+
+template <bool HM>
+optiml_status_t launch_umma2s_form(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
+                                   int K, int act, cudaStream_t st) {
+    using C = Umma2sCfgT<HM>;
     CUtensorMap ma, mb;
-    if (!get_map(h, &ma, A, (uint64_t)M, (uint64_t)K, 128, 64) || !get_map(h, &mb, B, (uint64_t)K, (uint64_t)N, 64, 64))
+    if (!get_map(h, &ma, A, (uint64_t)M, (uint64_t)K, C::kRowsPerCta, 64) || !get_map(h, &mb, B, (uint64_t)K, (uint64_t)N, 64, 64))
         return OPTIML_ERR_CUDA;
     Umma2sPlan plan;
     plan.tiles_m = (int)ceil_div64(M, C::BM);
@@ -514,18 +520,24 @@ optiml_status_t launch_umma2s(optiml_handle_t h, const void* A, const void* B, c
     plan.num_kb = (int)ceil_div64(K, C::BK);
     const int64_t tiles = (int64_t)plan.tiles_m * plan.tiles_n;
     plan.split = stream_split(h, tiles, plan.num_kb);
-    if (h->log) fprintf(stderr, "[optiml] streaming pair plan: tiles=%lld split=%d kb=%d\n", (long long)tiles, plan.split, plan.num_kb);
+    if (h->log) fprintf(stderr, "[optiml] streaming pair plan: %d-row tiles=%lld split=%d kb=%d\n", C::BM, (long long)tiles, plan.split, plan.num_kb);
     const int cluster = 2 * plan.split;
     const dim3 grid((unsigned)(tiles * cluster));
     const __nv_bfloat16* bi = (const __nv_bfloat16*)bias;
     switch (act) {
-    case OPTIML_ACT_RELU: launch_umma2s_act<kActRelu>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
-    case OPTIML_ACT_GELU_TANH: launch_umma2s_act<kActGeluTanh>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
-    case OPTIML_ACT_SIGMOID: launch_umma2s_act<kActSigmoid>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
-    default: launch_umma2s_act<kActNone>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
+    case OPTIML_ACT_RELU: launch_umma2s_act<kActRelu, HM>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
+    case OPTIML_ACT_GELU_TANH: launch_umma2s_act<kActGeluTanh, HM>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
+    case OPTIML_ACT_SIGMOID: launch_umma2s_act<kActSigmoid, HM>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
+    default: launch_umma2s_act<kActNone, HM>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
     }
     h->launches += 1;
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
+}
+
+optiml_status_t launch_umma2s(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
+                              int K, int act, cudaStream_t st) {
+    return stream_half_height(h, M) ? launch_umma2s_form<true>(h, A, B, bias, Y, M, N, K, act, st)
+                                    : launch_umma2s_form<false>(h, A, B, bias, Y, M, N, K, act, st);
 }
 
 // Clusters of `cluster` CTAs of the streaming pair kernel that can be resident at the same time.
@@ -542,7 +554,7 @@ int query_stream_clusters(int cluster) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_umma2s_kernel<kActNone>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_umma2s_kernel<kActNone, false>, &cfg) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -573,10 +585,14 @@ bool configure_kernels() {
     ok &= set_smem(gemm_umma2_kernel<kActRelu>, Umma2Cfg::kSmemBytes);
     ok &= set_smem(gemm_umma2_kernel<kActGeluTanh>, Umma2Cfg::kSmemBytes);
     ok &= set_smem(gemm_umma2_kernel<kActSigmoid>, Umma2Cfg::kSmemBytes);
-    ok &= set_smem(gemm_umma2s_kernel<kActNone>, Umma2sCfg::kSmemBytes);
-    ok &= set_smem(gemm_umma2s_kernel<kActRelu>, Umma2sCfg::kSmemBytes);
-    ok &= set_smem(gemm_umma2s_kernel<kActGeluTanh>, Umma2sCfg::kSmemBytes);
-    ok &= set_smem(gemm_umma2s_kernel<kActSigmoid>, Umma2sCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActNone, false>, Umma2sCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActRelu, false>, Umma2sCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActGeluTanh, false>, Umma2sCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActSigmoid, false>, Umma2sCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActNone, true>, Umma2sHalfCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActRelu, true>, Umma2sHalfCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActGeluTanh, true>, Umma2sHalfCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActSigmoid, true>, Umma2sHalfCfg::kSmemBytes);
     ok &= set_skinny(gemm_skinny_umma_kernel<16, 2>, SkinnyCfg<16, 2>::kSmemBytes);
     ok &= set_skinny(gemm_skinny_umma_kernel<16, 3>, SkinnyCfg<16, 3>::kSmemBytes);
     ok &= set_skinny(gemm_skinny_umma_kernel<32, 2>, SkinnyCfg<32, 2>::kSmemBytes);

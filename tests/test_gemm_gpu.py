@@ -109,6 +109,30 @@ def test_streaming_pair_variant(handle, M, N, K, act, split_max):
         handle.set_option(V.OPT_PAIR_SPLIT_MAX, 8)
 
 
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64),        # one tile, one K block
+                                   (128, 520, 1096),      # ragged columns and K, every lane of both halves live
+                                   (100, 264, 2048),      # rows 64..99 in the second CTA
+                                   (64, 1288, 520),       # the second CTA of every pair has no rows
+                                   (33, 776, 4096),
+                                   (5, 8, 8),
+                                   (96, 8192, 1024)])     # 32 tiles
+@pytest.mark.parametrize("act", [RELU, GELU])
+@pytest.mark.parametrize("split_max", [1, 2])
+def test_streaming_pair_variant_half_height_tiles(handle, M, N, K, act, split_max):
+    """M <= 128: 64 rows per CTA (tcgen05.mma.cta_group::2 with M = 128), on by default; the 256-row
+    form on the same shapes is the comparison."""
+    assert handle.get_option(V.OPT_PAIR_HALF_HEIGHT) == 1
+    handle.set_option(V.OPT_PAIR_SPLIT_MAX, split_max)
+    try:
+        c = synth.make_case("c4", M=M, N=N, K=K, act=act)
+        parity(handle, c, V.VARIANT_UMMA_2CTA_STREAM, "64 rows per CTA")
+        handle.set_option(V.OPT_PAIR_HALF_HEIGHT, 0)
+        parity(handle, c, V.VARIANT_UMMA_2CTA_STREAM, "128 rows per CTA")
+    finally:
+        handle.set_option(V.OPT_PAIR_SPLIT_MAX, 8)
+        handle.set_option(V.OPT_PAIR_HALF_HEIGHT, 1)
+
+
 def test_streaming_pair_variant_refuses_more_tiles_than_clusters(handle):
     handle.force_variant(V.VARIANT_UMMA_2CTA_STREAM)
     c = synth.make_case("c4", M=2048, N=4096, K=64)          # 128 tiles
@@ -149,7 +173,8 @@ def test_sigmoid_epilogue(handle, variant, name, M, N, K):
     (V.VARIANT_GEMV_SPLITK, BF16, 4, 520, 1000), (V.VARIANT_SKINNY_UMMA, BF16, 16, 1160, 1096),
     (V.VARIANT_SKINNY_UMMA, BF16, 48, 648, 2048), (V.VARIANT_UMMA, BF16, 384, 776, 1024),
     (V.VARIANT_UMMA_2CTA, BF16, 384, 776, 1024), (V.VARIANT_UMMA_2CTA, BF16, 1000, 520, 320),
-    (V.VARIANT_UMMA_2CTA_STREAM, BF16, 384, 776, 1024), (V.VARIANT_UMMA_2CTA_STREAM, BF16, 100, 2056, 4096)])
+    (V.VARIANT_UMMA_2CTA_STREAM, BF16, 384, 776, 1024), (V.VARIANT_UMMA_2CTA_STREAM, BF16, 100, 2056, 4096),
+    (V.VARIANT_UMMA_2CTA_STREAM, BF16, 128, 776, 1024)])
 @pytest.mark.parametrize("act", [NONE, RELU])
 def test_integer_inputs_are_bit_exact(handle, variant, dtype, M, N, K, act):
     c = synth.integer_case(M, N, K, dtype, act, seed=11)
@@ -293,6 +318,7 @@ def test_dispatcher_choices(handle):
     assert sel(32, 4096, 4096, BF16) == V.VARIANT_SKINNY_UMMA and sel(2, 4096, 4096, BF16) == V.VARIANT_SKINNY_UMMA
     assert sel(64, 14336, 4096, BF16) == V.VARIANT_SKINNY_UMMA          # every column tile whole in one CTA
     assert sel(64, 8192, 8192, BF16) == V.VARIANT_UMMA_2CTA_STREAM      # the skinny schedule would cut tiles along K
+    assert sel(96, 14336, 4096, BF16) == V.VARIANT_UMMA_2CTA_STREAM     # above 64 rows the cluster kernel (64 rows per CTA)
     assert sel(130, 262, 100, BF16) == V.VARIANT_GENERIC         # N % 8 != 0 (large ones are re-pitched, then dispatched again)
     assert sel(0, 1, 1, BF16) == -1
 
