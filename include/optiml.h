@@ -67,9 +67,9 @@ typedef enum {
     OPTIML_VARIANT_SKINNY_UMMA = 3, /* bf16, M <= 128: stream-K over B with tcgen05 (N is the MMA M dim) */
     OPTIML_VARIANT_UMMA = 4,        /* bf16: persistent TMA + tcgen05 + TMEM tiles, N % 8 == K % 8 == 0  */
     OPTIML_VARIANT_UMMA_2CTA = 5,   /* bf16: the same with CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles) */
-    OPTIML_VARIANT_UMMA_2CTA_STREAM = 6, /* bf16, fewer 256 x 256 tiles than CTA pairs: one cluster of 2, 4 or 8 CTAs per
-                                            tile, K cut across its CTA pairs, partial sums exchanged through
-                                            distributed shared memory                                         */
+    OPTIML_VARIANT_UMMA_2CTA_STREAM = 6, /* bf16, fewer tiles than CTA pairs: one cluster of 2 or 4 CTAs per tile
+                                            (256 x 256; 128 x 256 with 64 rows per CTA for M <= 128), K cut across
+                                            its CTA pairs, partial sums exchanged through distributed shared memory */
     OPTIML_VARIANT_COUNT = 7
 } optiml_variant_t;
 
