@@ -82,12 +82,13 @@ inline UmmaPlan make_umma2_plan(int64_t M, int64_t N, int64_t K, int num_sms, in
 }
 
 // i-th work item of CTA pair `c`; tile coordinates in units of 256 x 256.
-__device__ __forceinline__ bool umma2_work_item(const UmmaPlan& p, int c, int i, UmmaWork& w) {
+__host__ __device__ __forceinline__ bool umma2_work_item(const UmmaPlan& p, int c, int i, UmmaWork& w) {
     auto coords = [&](int t, int& tm, int& tn) {
         const int group_size = Umma2Cfg::kGroupM * p.tiles_n;
         const int group = t / group_size;
         const int first_m = group * Umma2Cfg::kGroupM;
-        const int rows = min(Umma2Cfg::kGroupM, p.tiles_m - first_m);
+        const int left = p.tiles_m - first_m;
+        const int rows = left < Umma2Cfg::kGroupM ? left : Umma2Cfg::kGroupM;
         const int in_group = t - group * group_size;
         tm = first_m + in_group % rows;
         tn = in_group / rows;

@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "kernel_skinny.cuh"
+#include "kernel_umma2.cuh"
 
 using namespace optiml;
 
@@ -49,7 +50,70 @@ static int check(int64_t T, int64_t KB, int sms, int64_t max_slots) {
     return 0;
 }
 
+// The persistent CTA-pair kernel's work split: whole tiles round-robin, the tiles of the last
+// partial round cut into K slices, one slice per pair.  Every (tile, K block) must be covered
+// exactly once and every cut tile by exactly `split` slices with distinct indices.
+static int check_pair_plan(int64_t M, int64_t N, int64_t K, int sms, int split_max) {
+    const UmmaPlan p = make_umma2_plan(M, N, K, sms, split_max);
+    const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
+    if (p.grid < 1 || p.grid > sms / 2 || p.split < 1 || p.split > split_max) return 1;
+    if (p.split == 1 ? (p.rem_tiles != 0 || p.full_tiles != tiles) : (p.full_tiles + p.rem_tiles != tiles)) return 2;
+    if ((int64_t)p.rem_tiles * p.split > sms / 2) return 3;      // one slice per pair
+    std::vector<int> cover((size_t)(tiles * p.num_kb), 0);
+    std::set<std::pair<int, int>> slices;
+    int most_items = 0;
+    for (int c = 0; c < p.grid; ++c) {
+        UmmaWork w;
+        int i = 0;
+        for (; umma2_work_item(p, c, i, w); ++i) {
+            if (w.tm < 0 || w.tm >= p.tiles_m || w.tn < 0 || w.tn >= p.tiles_n || w.kb0 < 0 || w.kb0 >= w.kb1 || w.kb1 > p.num_kb)
+                return 4;
+            if (w.rem_idx >= 0) {
+                if (w.rem_idx >= p.rem_tiles || w.chunk < 0 || w.chunk >= p.split) return 5;
+                if (!slices.insert({w.rem_idx, w.chunk}).second) return 6;
+            } else if (w.kb0 != 0 || w.kb1 != p.num_kb) {
+                return 7;
+            }
+            for (int kb = w.kb0; kb < w.kb1; ++kb) cover[((size_t)w.tn * p.tiles_m + w.tm) * p.num_kb + kb] += 1;
+            if (i > 1 << 20) return 8;
+        }
+        if (i > most_items) most_items = i;
+    }
+    for (int v : cover)
+        if (v != 1) return 9;
+    if ((int64_t)slices.size() != (int64_t)p.rem_tiles * p.split) return 10;
+    // at most one slice after a pair's whole tiles
+    const int64_t whole_rounds = (p.full_tiles + p.grid - 1) / p.grid;
+    if (most_items > whole_rounds + 1) return 11;
+    return 0;
+}
+
 int main() {
+    {
+        int bad_pairs = 0, n_pairs = 0;
+        const int64_t Ms[] = {1, 256, 257, 512, 1024, 2304, 4096, 8192}, Ns[] = {8, 256, 520, 4096, 8192, 14336, 28672};
+        const int64_t Ks[] = {8, 64, 256, 1032, 4096, 16384};
+        for (int64_t M : Ms)
+            for (int64_t N : Ns)
+                for (int64_t K : Ks)
+                    for (int sms : {2, 16, 132, 148})
+                        for (int split_max : {1, 2, 3, 8}) {
+                            const int rc = check_pair_plan(M, N, K, sms, split_max);
+                            ++n_pairs;
+                            if (rc) {
+                                std::printf("FAIL pair plan M=%lld N=%lld K=%lld sms=%d split_max=%d code=%d\n", (long long)M,
+                                            (long long)N, (long long)K, sms, split_max, rc);
+                                ++bad_pairs;
+                            }
+                        }
+        // 512 x 14336 x 4096 on 74 pairs: 112 whole tiles in two rounds (38 tiles cannot be cut for 74 pairs);
+        // 4096^3: 222 whole tiles, 34 tiles in 2 slices
+        const UmmaPlan a = make_umma2_plan(512, 14336, 4096, 148, 8), b = make_umma2_plan(4096, 4096, 4096, 148, 8);
+        std::printf("pair plan 512x14336x4096: full=%d rem=%d split=%d grid=%d; 4096^3: full=%d rem=%d split=%d grid=%d\n", a.full_tiles,
+                    a.rem_tiles, a.split, a.grid, b.full_tiles, b.rem_tiles, b.split, b.grid);
+        std::printf("%d pair plans checked, %d wrong\n", n_pairs, bad_pairs);
+        if (bad_pairs) return 1;
+    }
     const int64_t Ts[] = {1, 2, 3, 7, 37, 56, 64, 73, 74, 75, 111, 112, 147, 148, 149, 160, 200, 296, 300, 1000, 5000};
     const int64_t KBs[] = {1, 2, 3, 5, 16, 17, 63, 64, 65, 128, 257};
     const int smss[] = {1, 2, 7, 132, 148};

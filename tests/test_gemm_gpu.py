@@ -85,6 +85,7 @@ def test_skinny_variant(handle, M, N, K, act):
                                    (1024, 1024, 512),     # 32 tiles: each cut into 2 K slices
                                    (256, 520, 4096),      # 6 tiles, 8 K slices each
                                    (2432, 4096, 256),     # 304 tiles = 2 rounds + 8 tiles cut into 4 K slices
+                                   (512, 14336, 520),     # 112 tiles on 74 CTA pairs: two rounds of whole tiles
                                    (2048, 4096, 128)])   # 256 tiles: more than one tile per CTA
 @pytest.mark.parametrize("act", [RELU, GELU])
 @pytest.mark.parametrize("variant", [V.VARIANT_UMMA, V.VARIANT_UMMA_2CTA])
@@ -262,14 +263,17 @@ def test_c4_c5_sampled(handle, name):
     assert np.array_equal(bits, bits2)
 
 
-@pytest.mark.parametrize("M,N,K", [(256, 8192, 8192),      # 32 tiles, two CTA pairs per tile: the exchange between the pairs
-                                   (128, 8192, 8192),      # the same with an empty second CTA in every pair
-                                   (256, 14336, 4096),     # 56 tiles, one pair per tile
-                                   (512, 8192, 8192)])     # two rows of tiles
-def test_crossover_shapes_of_the_cluster_kernel_on_sampled_outputs(handle, M, N, K):
+@pytest.mark.parametrize("M,N,K,variant", [
+    (256, 8192, 8192, V.VARIANT_UMMA_2CTA_STREAM),      # 32 tiles, two CTA pairs per tile: the exchange between the pairs
+    (128, 8192, 8192, V.VARIANT_UMMA_2CTA_STREAM),      # the same with 128-row tiles, 64 rows per CTA
+    (96, 14336, 4096, V.VARIANT_UMMA_2CTA_STREAM),      # 128-row tiles, one pair per tile, rows 64..95 in the second CTA
+    (256, 14336, 4096, V.VARIANT_UMMA_2CTA_STREAM),     # 56 tiles, one pair per tile
+    (512, 8192, 8192, V.VARIANT_UMMA_2CTA_STREAM),      # two rows of tiles
+    (512, 14336, 4096, V.VARIANT_UMMA_2CTA)])           # persistent pairs: two rounds of whole tiles, the second half empty
+def test_crossover_shapes_on_sampled_outputs(handle, M, N, K, variant):
     """The shapes of the dispatcher's crossover table at full size, as the benchmark launches them."""
     c = synth.make_case("c4", M=M, N=N, K=K)
-    assert handle.select_variant(M, N, K, c.dtype) == V.VARIANT_UMMA_2CTA_STREAM
+    assert handle.select_variant(M, N, K, c.dtype) == variant
     bits, y = H.run_case(handle, c)
     rows = sample_indices(M, 128, 96, 1)
     cols = sample_indices(N, 256, 320, 2)
