@@ -216,15 +216,21 @@ class Timer:
             self.i += 1
         torch.cuda.synchronize(self.device)
 
-    def region(self, launches, barrier=False):
+    def region(self, launches, barrier=False, gate=None):
         """`launches` back-to-back calls between two events -> (milliseconds, host t0, host t1).
-        (An event after every call would put 3-4 us of idle time between consecutive kernels.)"""
+        (An event after every call would put 3-4 us of idle time between consecutive kernels.)
+        With `gate` (a callable that enqueues a short busy kernel) the first event is recorded behind
+        that kernel, so the first calls are already queued when the event completes: a region of a
+        few launches then holds the launches and nothing of the host's start-up (about 10 us between
+        an event record and the first launch reaching an idle GPU from Python)."""
         torch.cuda.synchronize(self.device)
         if barrier:
             replicas.barrier()
             torch.cuda.synchronize(self.device)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0 = time.perf_counter()
+        if gate is not None:
+            gate()
         e0.record(self.stream)
         for _ in range(launches):
             self.step(self.i)
@@ -424,8 +430,10 @@ def measure_once(handle, name, case, bound, args, sampler, device, peaks, peak_s
     if contract_steps:
         # the headline region: W warm-up steps, exactly K steps, barrier + synchronize on both sides
         timer.warm(args.warmup)
-        ms, t0, t1 = timer.region(contract_steps, barrier=True)
+        ms_host, _, _ = timer.region(contract_steps, barrier=True)
+        ms, t0, t1 = timer.region(contract_steps, barrier=True, gate=make_gate(device))
         out["contract_ms"], out["contract_steps"] = ms, contract_steps
+        out["contract_ms_host_started"] = ms_host
         out["contract_clocks"] = timer.clocks(t0, t1)
     min_l = PROTOCOL_MIN_LAUNCHES.get(name, 20)
     stats, t0, t1 = protocol(timer, min_l if not quick else min(min_l, 20), estimate_ms(case, bound, peaks))
@@ -839,6 +847,13 @@ def main():
             "gpu_launches": args.steps, "gpu_launches_all_legs": main_res["launches"],
             "replicas": "independent replicas, no data-path collective",
             "per_shape": per_shape, "reductions": reductions, "attention": attention, "extra_shapes": extras}
+    line["timed_region"] = {
+        "how": "W warm-up steps, barrier + synchronize, a busy kernel of about 60 us, start event, exactly K steps, end "
+               "event, synchronize + barrier: the K launches are queued behind the busy kernel when the start event "
+               "completes, so the region holds the K steps and none of the host's start-up",
+        "ms_per_step_host_started": main_res["contract_ms_host_started"] / args.steps,
+        "host_started": "the same K steps with the start event recorded on an idle GPU, i.e. including the time the "
+                        "host needs to get the first launch there (this rank's figure)"}
     if "single_call_us" in main_res:
         line["single_call_us"] = main_res["single_call_us"]
         line["single_call_floor_us"] = isolated_floor_us(handle, device, sampler)
