@@ -233,13 +233,15 @@ int choose_variant(optiml_handle_t h, int64_t M, int64_t N, int64_t K, int dtype
     if (M == 1 && variant_supports(h, OPTIML_VARIANT_GEMV_SPLITK, M, N, K, dtype, al16)) return OPTIML_VARIANT_GEMV_SPLITK;
     const bool skinny_ok = variant_supports(h, OPTIML_VARIANT_SKINNY_UMMA, M, N, K, dtype, al16);
     const bool stream_ok = variant_supports(h, OPTIML_VARIANT_UMMA_2CTA_STREAM, M, N, K, dtype, al16);
+    // up to 32 rows the stream-K kernel spreads any shape over all SMs (4096 x 14336 with 16 column tiles of 256:
+    // 32 rows 25.5 us against 33.1 us for the cluster kernel, which has 64 CTAs there; 8192 x 8192: 25.8 against 25.0 us)
     if (M <= 32 && skinny_ok) return OPTIML_VARIANT_SKINNY_UMMA;
     if (M <= 128 && skinny_ok) {
         // Between 33 and 128 rows the streaming kernel with N as the MMA M dimension wins up to 64 rows where
-        // every column tile is finished by one CTA (measured 64 x 14336 x 4096: 21.9 us against 23.0 us for
-        // the cluster kernel with 64 rows per CTA), and loses above (128 rows: 25.7 against 23.7 us) and
-        // wherever its tiles are cut along K (64 x 8192 x 8192: 31.3 against 25.5 us; 128 rows: 41.4
-        // against 25.6 us).
+        // every column tile is finished by one CTA (measured 64 x 14336 x 4096: 21.4 us against 23.0 us for
+        // the cluster kernel with 64 rows per CTA), and loses above (128 rows: 25.3 against 23.4 us) and
+        // wherever its tiles are cut along K (48 x 8192 x 8192: 28.8 against 25.2 us; 64 rows: 31.2 against
+        // 25.5 us; 128 rows: 41.5 against 25.5 us; 48 x 2048 x 8192: 38.3 against 20.8 us).
         if (!stream_ok || (M <= 64 && skinny_single_band(h, M, N, K))) return OPTIML_VARIANT_SKINNY_UMMA;
         return OPTIML_VARIANT_UMMA_2CTA_STREAM;
     }
