@@ -67,7 +67,7 @@ typedef enum {
     OPTIML_VARIANT_SKINNY_UMMA = 3, /* bf16, M <= 128: stream-K over B with tcgen05 (N is the MMA M dim) */
     OPTIML_VARIANT_UMMA = 4,        /* bf16: persistent TMA + tcgen05 + TMEM tiles, N % 8 == K % 8 == 0  */
     OPTIML_VARIANT_UMMA_2CTA = 5,   /* bf16: the same with CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles) */
-    OPTIML_VARIANT_UMMA_2CTA_STREAM = 6, /* bf16, fewer tiles than CTA pairs: one cluster of 2 or 4 CTAs per tile
+    OPTIML_VARIANT_UMMA_2CTA_STREAM = 6, /* bf16, fewer tiles than CTA pairs: one cluster of 2, 4 or 8 CTAs per tile
                                             (256 x 256; 128 x 256 with 64 rows per CTA for M <= 128), K cut across
                                             its CTA pairs, partial sums exchanged through distributed shared memory */
     OPTIML_VARIANT_COUNT = 7
@@ -283,7 +283,7 @@ typedef enum {
     OPTIML_OPT_SKINNY_LATE_TRIGGER = 4,   /* skinny: 1 = release the next kernel's CTAs after a CTA's last load,
                                              0 = as soon as the kernel starts                                       */
     OPTIML_OPT_PAIR_SPLIT_MAX = 5,        /* CTA-pair GEMMs: most K slices a tile is cut into (persistent form: tiles of
-                                             the last, partial round, up to 8; streaming form: 1 or 2)          */
+                                             the last, partial round, up to 8; streaming form: 1, 2 or 4)          */
     OPTIML_OPT_PAIR_HALF_HEIGHT = 6,      /* streaming CTA-pair form, M <= 128: 1 = 128-row tiles, 64 rows per CTA
                                              (default), 0 = 256-row tiles as for larger M                            */
     OPTIML_OPT_COUNT = 7

@@ -3,7 +3,7 @@
 // one tile row only, so the problem is a stream over B, and what decides the time is how many
 // SMs pull on that stream and how short the fixed part around the main loop is.
 //
-// One thread-block cluster of 2 S CTAs (S = 1 or 2) per tile.  The cluster holds S CTA pairs
+// One thread-block cluster of 2 S CTAs (S = 1, 2 or 4) per tile.  The cluster holds S CTA pairs
 // ("bands"); band b computes the tile over K blocks [KB b / S, KB (b + 1) / S) with
 // tcgen05.mma.cta_group::2 exactly as the persistent CTA-pair kernel does (each CTA stages its
 // own 128 rows of A and 128 columns of B with plain TMA loads; no load is shared between CTAs).
@@ -16,7 +16,10 @@
 // bias + activation and stores its 128 x 128 block of Y: a reduce-scatter, so the
 // epilogue is halved as well, nothing goes through global scratch and nothing is counted with
 // atomics.  (Writing the partner's ring with ordinary remote stores instead took 2.8 us for the
-// 64 KiB.)
+// 64 KiB.)  With S = 4 (shapes of at most 18 tiles or so, where two pairs per tile would leave
+// half of the SMs idle) the same happens among four CTAs: each keeps a quarter of its columns,
+// sends the other three quarters to the three CTAs with the same h and adds four shares in band
+// order.
 //
 //   warp 0      TMA producer (one lane), as in kernel_umma2.cuh
 //   warp 1      tensor-memory allocation (256 columns, cta_group::2); MMA-issuing lane in the
@@ -64,7 +67,7 @@ struct Umma2sCfgT {
     static_assert(kStageBytes % 1024 == 0, "swizzle atoms start on 1024-byte boundaries");
     static_assert(kSendOffset + kShareBytes <= kRingBytes, "ring reuse");
     static constexpr int kSmemBytes = kRingBytes + 256 + 1024;
-    static constexpr int kMaxSplit = 2;                      // cluster of 4 CTAs
+    static constexpr int kMaxSplit = 4;                      // cluster of 8 CTAs
 };
 using Umma2sCfg = Umma2sCfgT<false>;
 using Umma2sHalfCfg = Umma2sCfgT<true>;
@@ -82,8 +85,8 @@ struct Umma2sShared {
     uint64_t empty[kUmma2sMaxStages];      // per CTA, signalled by the leader's commit
     uint64_t tmem_full;                    // per CTA, signalled by the leader's commit
     uint64_t drain;
-    uint64_t partner_idle;                 // the partner's main loop is over: its ring may be written
-    uint64_t recv_full;                    // the partner's share has landed in this CTA's ring
+    uint64_t partner_idle;                 // the partners' main loops are over (S - 1 arrivals): their rings may be written
+    uint64_t recv_full;                    // the partners' shares have landed in this CTA's ring
     uint32_t tmem_base;
     volatile int abort;
 };
@@ -141,12 +144,12 @@ gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         }
         ptx::mbar_init(&sh->tmem_full, 1);
         ptx::mbar_init(&sh->drain, 1);
-        ptx::mbar_init(&sh->partner_idle, 1);
+        ptx::mbar_init(&sh->partner_idle, S > 1 ? S - 1 : 1);
         ptx::mbar_init(&sh->recv_full, 1);
         sh->abort = 0;
         ptx::fence_mbar_init();
         // the partner's copy may complete at any time after the cluster barrier below
-        if (S > 1) ptx::mbar_arrive_expect_tx(&sh->recv_full, C::kShareBytes);
+        if (S > 1) ptx::mbar_arrive_expect_tx(&sh->recv_full, (uint32_t)((S - 1) * (128 * (C::kTmemCols / S) * 4)));
     }
     if (warp == 1) {
         ptx::tmem_alloc_2cta(&sh->tmem_base, C::kTmemCols);
@@ -228,6 +231,136 @@ gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             ptx::umma_commit_2cta_local(&sh->drain);
             ptx::mbar_wait(&sh->drain, 0);
         }
+    } else if (S > 2) {
+        // ------------------------------------------------------------ epilogue warps, more than two bands
+        // Tensor-memory lane L of this CTA holds one row of the tile in its kTmemCols columns (256-row
+        // tiles: row L, columns 0..255; 128-row tiles: row L % 64, columns [128 (L / 64), +128)).  Band b
+        // finishes columns [keep b, keep b + keep) of every lane, keep = kTmemCols / S, and sends chunk d
+        // to the CTA of band d with the same h.  A share is 128 lanes x keep columns of fp32, float4
+        // index (column / 4) * 128 + lane; the ring holds S - 1 received shares, then S - 1 outgoing
+        // ones.  Of the two warps on a lane quarter each takes half of every chunk, 16 columns at a time.
+        constexpr int CT = C::kTmemCols;
+        const int ew = warp - 2, q = warp & 3, ch = ew >> 2;
+        const int L = q * 32 + lane;
+        const int keep = CT / S, W = keep / 2, ng = W / 16;        // 256-row tiles, S = 4: 64, 32, 2; 128-row tiles: 32, 16, 1
+        const uint32_t share_bytes = (uint32_t)(128 * keep * 4);
+        const uint32_t recv_off = 0, send_off = (uint32_t)(S - 1) * share_bytes;
+        const bool rows_live = (int64_t)tm * C::BM + hc * C::kRowsPerCta < M;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
+        const int64_t m = (int64_t)tm * C::BM + hc * C::kRowsPerCta + (HM ? (L & 63) : L);
+        const int64_t n0 = (int64_t)tn * C::BN + (HM ? (q >> 1) * 128 : 0) + band * keep + ch * W;   // first column of Y of this thread
+        auto slot_of = [](int other, int self) { return other < self ? other : other - 1; };   // index among the S - 1 others
+
+        uint4 bias_w[2][2];                                 // fetched while the main loop runs
+#pragma unroll
+        for (int g = 0; g < 2; ++g)
+#pragma unroll
+            for (int v = 0; v < 2; ++v) {
+                const int64_t n = n0 + g * 16 + v * 8;
+                bias_w[g][v] = (bias && g < ng && n < N) ? *reinterpret_cast<const uint4*>(bias + n)   // N % 8 == 0
+                                                         : make_uint4(0, 0, 0, 0);
+            }
+
+        bool ok = (kb1 > kb0) && !sh->abort && ptx::mbar_wait(&sh->tmem_full, 0);
+        ok = __all_sync(0xffffffffu, ok);
+        int site = 5;
+        ptx::tcgen05_fence_after_sync();
+
+        if (ok && threadIdx.x == 64) {
+            for (int d = 0; d < S; ++d)
+                if (d != band) ptx::mbar_arrive_cluster(ptx::mapa_shared(ptx::smem_u32(&sh->partner_idle), (uint32_t)(2 * d + hc)));
+        }
+        if (ok && rows_live) {
+            for (int d = 0; d < S; ++d) {
+                if (d == band) continue;
+                float4* send = reinterpret_cast<float4*>(ring + send_off + (uint32_t)slot_of(d, band) * share_bytes) + L;
+                for (int g = 0; g < ng; ++g) {
+                    uint32_t r[16];
+                    ptx::tmem_ld_32x16(t_lane + d * keep + ch * W + g * 16, r);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int v = 0; v < 4; ++v)
+                        send[((ch * W + g * 16) / 4 + v) * 128] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                                              __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                }
+            }
+            ptx::fence_proxy_async_smem();
+        }
+        umma2s_epi_bar_sync();
+        if (threadIdx.x == 64 && ok && rows_live) {
+            if (ptx::mbar_wait(&sh->partner_idle, 0)) {
+                for (int d = 0; d < S; ++d) {
+                    if (d == band) continue;
+                    const uint32_t peer = (uint32_t)(2 * d + hc);
+                    bulk_copy_to_cluster(ptx::mapa_shared(ring_base + recv_off + (uint32_t)slot_of(band, d) * share_bytes, peer),
+                                         ring + send_off + (uint32_t)slot_of(d, band) * share_bytes, share_bytes,
+                                         ptx::mapa_shared(ptx::smem_u32(&sh->recv_full), peer));
+                }
+            } else {
+                site = 8;
+            }
+        }
+
+        uint32_t racc[2][16];
+        if (ok && rows_live) {
+#pragma unroll
+            for (int g = 0; g < 2; ++g)
+                if (g < ng) ptx::tmem_ld_32x16(t_lane + band * keep + ch * W + g * 16, racc[g]);
+        }
+        if (ok && rows_live && !ptx::mbar_wait(&sh->recv_full, 0)) {
+            ok = false;
+            site = 9;
+        }
+        ok = __all_sync(0xffffffffu, ok);
+
+        if (ok && rows_live) {
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+                if (g >= ng) break;
+                float x[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) x[i] = 0.0f;
+                // shares in band order = ascending K, this CTA's own among them
+                for (int sb = 0; sb < S; ++sb) {
+                    if (sb == band) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) x[i] += __uint_as_float(racc[g][i]);
+                    } else {
+                        const float4* recv = reinterpret_cast<const float4*>(ring + recv_off + (uint32_t)slot_of(sb, band) * share_bytes) + L;
+                        float4 t[4];
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) t[v] = recv[((ch * W + g * 16) / 4 + v) * 128];
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            x[4 * v] += t[v].x;
+                            x[4 * v + 1] += t[v].y;
+                            x[4 * v + 2] += t[v].z;
+                            x[4 * v + 3] += t[v].w;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int v = 0; v < 2; ++v) {
+                    const int64_t n = n0 + g * 16 + v * 8;
+                    const uint4 bw = bias_w[g][v];
+                    const uint32_t bwv[4] = {bw.x, bw.y, bw.z, bw.w};
+                    uint32_t o[4];
+#pragma unroll
+                    for (int p = 0; p < 4; ++p) {
+                        const float y0 = epilogue<ACT, true>(x[v * 8 + 2 * p], bf16lo_to_f32(bwv[p]));
+                        const float y1 = epilogue<ACT, true>(x[v * 8 + 2 * p + 1], bf16hi_to_f32(bwv[p]));
+                        o[p] = pack_bf16x2(y0, y1);
+                    }
+                    if (m < M && n < N) *reinterpret_cast<uint4*>(Y + m * N + n) = make_uint4(o[0], o[1], o[2], o[3]);
+                }
+            }
+        }
+        if (!ok && lane == 0 && kb1 > kb0) {
+            report_timeout(status, site);
+            sh->abort = 1;
+        }
+        if (site == 8) report_timeout(status, 8);
     } else if constexpr (!HM) {
         // ------------------------------------------------------------ epilogue warps
         const int ew = warp - 2;                            // 0..7 among the epilogue warps

@@ -118,7 +118,7 @@ struct optiml_handle_s {
     void* pad[4] = {nullptr, nullptr, nullptr, nullptr};       // re-pitched copies of A, B, bias, Y (unaligned bf16 shapes)
     size_t pad_bytes[4] = {0, 0, 0, 0};
     int64_t options[OPTIML_OPT_COUNT];
-    int stream_clusters[2] = {0, 0};      // clusters of 2 and of 4 CTAs of the streaming pair kernel the device can hold at once
+    int stream_clusters[3] = {0, 0, 0};   // clusters of 2, 4 and 8 CTAs of the streaming pair kernel the device can hold at once
 };
 
 namespace {
@@ -739,8 +739,8 @@ optiml_status_t optiml_create(optiml_handle_t* out, int device) {
     ok = ok && cudaMemset(h->status, 0, sizeof(int)) == cudaSuccess;
     ok = ok && configure_kernels();
     if (ok)
-        for (int i = 0; i < 2; ++i) h->stream_clusters[i] = query_stream_clusters(2 << i);
-    if (h->log) fprintf(stderr, "[optiml] resident clusters of the streaming pair kernel: %d of 2 CTAs, %d of 4 CTAs\n", h->stream_clusters[0], h->stream_clusters[1]);
+        for (int i = 0; i < 3; ++i) h->stream_clusters[i] = query_stream_clusters(2 << i);
+    if (h->log) fprintf(stderr, "[optiml] resident clusters of the streaming pair kernel: %d of 2 CTAs, %d of 4, %d of 8\n", h->stream_clusters[0], h->stream_clusters[1], h->stream_clusters[2]);
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) {
         cudaGetLastError();

@@ -118,7 +118,7 @@ def test_streaming_pair_variant(handle, M, N, K, act, split_max):
                                    (5, 8, 8),
                                    (96, 8192, 1024)])     # 32 tiles
 @pytest.mark.parametrize("act", [RELU, GELU])
-@pytest.mark.parametrize("split_max", [1, 2])
+@pytest.mark.parametrize("split_max", [1, 2, 4])
 def test_streaming_pair_variant_half_height_tiles(handle, M, N, K, act, split_max):
     """M <= 128: 64 rows per CTA (tcgen05.mma.cta_group::2 with M = 128), on by default; the 256-row
     form on the same shapes is the comparison."""
