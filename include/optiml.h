@@ -286,7 +286,9 @@ typedef enum {
                                              the last, partial round, up to 8; streaming form: 1, 2 or 4)          */
     OPTIML_OPT_PAIR_HALF_HEIGHT = 6,      /* streaming CTA-pair form, M <= 128: 1 = 128-row tiles, 64 rows per CTA
                                              (default), 0 = 256-row tiles as for larger M                            */
-    OPTIML_OPT_COUNT = 7
+    OPTIML_OPT_PAIR_TILE_WIDTH = 7,       /* streaming CTA-pair form: 0 = tile width chosen per shape (default),
+                                             128 or 256 = that width                                                 */
+    OPTIML_OPT_COUNT = 8
 } optiml_option_t;
 optiml_status_t optiml_set_option(optiml_handle_t h, optiml_option_t opt, int64_t value);
 int64_t optiml_get_option(optiml_handle_t h, optiml_option_t opt);

@@ -22,8 +22,8 @@ VARIANT_COUNT = 7
 REDUCE_SUM, REDUCE_DOT, REDUCE_MSE = 0, 1, 2
 
 (OPT_GEMV_PREFETCH_ROWS, OPT_SKINNY_STAGE_ROWS, OPT_SKINNY_RING_STAGES, OPT_SKINNY_PREFETCH_EARLY,
- OPT_SKINNY_LATE_TRIGGER, OPT_PAIR_SPLIT_MAX, OPT_PAIR_HALF_HEIGHT) = range(7)
-OPT_COUNT = 7
+ OPT_SKINNY_LATE_TRIGGER, OPT_PAIR_SPLIT_MAX, OPT_PAIR_HALF_HEIGHT, OPT_PAIR_TILE_WIDTH) = range(8)
+OPT_COUNT = 8
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ARCH, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(8)
 

@@ -47,33 +47,39 @@ namespace optiml {
 // work.  The accumulator of a CTA then sits in tensor memory as lanes [0, 64) = its 64 rows x
 // columns [0, 128) of the tile and lanes [64, 128) = the same rows x columns [128, 256):
 // 128 tensor-memory columns in all.
-template <bool HM>
+// BN_ = 128 (the "narrow" form): tiles of 128 columns, 64 per CTA, for shapes whose 256-column
+// tiles are too few to give every SM a CTA even with the K split (N = 4096: 16 tiles).
+template <bool HM, int BN_ = 256>
 struct Umma2sCfgT {
-    static constexpr int BM = HM ? 128 : 256, BN = 256, BK = 64, kStages = HM ? 8 : 6;
+    static_assert(BN_ == 256 || BN_ == 128, "tile width");
+    static constexpr int BM = HM ? 128 : 256, BN = BN_, BK = 64;
     static constexpr int kRowsPerCta = BM / 2;
     static constexpr int kABytes = kRowsPerCta * 64 * 2;     // this CTA's rows x 64 k of A
     static constexpr int kBChunkBytes = 64 * 64 * 2;         // 64 k x 64 columns
-    static constexpr int kBBytes = 2 * kBChunkBytes;         // 64 k x this CTA's 128 columns of B
-    static constexpr int kStageBytes = kABytes + kBBytes;    // 32 KiB (24 KiB)
+    static constexpr int kBChunks = BN / 128;                // 64-column chunks of B per CTA
+    static constexpr int kBBytes = kBChunks * kBChunkBytes;  // 64 k x this CTA's half of the tile's columns
+    static constexpr int kStageBytes = kABytes + kBBytes;    // 32, 24 or 16 KiB
+    static constexpr int kStages = 196608 / kStageBytes;     // a 192 KiB ring: 6, 8 or 12 stages
     static constexpr int kEpiWarps = 8;
     static constexpr int kThreads = 64 + 32 * kEpiWarps;
-    static constexpr int kTmemCols = HM ? 128 : 256;
-    // After the main loop the ring is reused: one share (the half of this CTA's accumulator that
-    // the partner finishes: 128 rows x 128 columns of fp32, or 64 x 128) is received, one is held
-    // on its way to the partner.
-    static constexpr int kShareBytes = kRowsPerCta * 128 * 4;
+    static constexpr int kTmemCols = HM ? BN / 2 : BN;       // accumulator columns per lane
+    // After the main loop the ring is reused: with two pairs per tile one share (the half of this
+    // CTA's accumulator that the partner finishes) is received, one is held on its way to the partner.
+    static constexpr int kShareBytes = 128 * (kTmemCols / 2) * 4;
     static constexpr int kRecvOffset = 0, kSendOffset = kShareBytes;
     static constexpr int kRingBytes = kStages * kStageBytes;
     static_assert(kStageBytes % 1024 == 0, "swizzle atoms start on 1024-byte boundaries");
-    static_assert(kSendOffset + kShareBytes <= kRingBytes, "ring reuse");
+    // S pairs per tile: S - 1 received and S - 1 outgoing shares of 128 lanes x (kTmemCols / S) columns
+    static_assert(2 * 3 * 128 * (kTmemCols / 4) * 4 <= kRingBytes && kSendOffset + kShareBytes <= kRingBytes, "ring reuse");
     static constexpr int kSmemBytes = kRingBytes + 256 + 1024;
     static constexpr int kMaxSplit = 4;                      // cluster of 8 CTAs
 };
 using Umma2sCfg = Umma2sCfgT<false>;
 using Umma2sHalfCfg = Umma2sCfgT<true>;
-static_assert(Umma2sCfg::kSmemBytes == Umma2sHalfCfg::kSmemBytes && Umma2sCfg::kThreads == Umma2sHalfCfg::kThreads,
-              "both forms launch alike (the resident-cluster counts are queried once)");
-constexpr int kUmma2sMaxStages = 8;
+static_assert(Umma2sCfg::kSmemBytes >= Umma2sHalfCfg::kSmemBytes && Umma2sCfg::kSmemBytes >= Umma2sCfgT<false, 128>::kSmemBytes &&
+              Umma2sCfg::kSmemBytes >= Umma2sCfgT<true, 128>::kSmemBytes && Umma2sCfg::kThreads == Umma2sHalfCfg::kThreads,
+              "the resident-cluster counts are queried once, for the form that needs most shared memory");
+constexpr int kUmma2sMaxStages = 12;
 
 struct Umma2sPlan {
     int tiles_m, tiles_n, num_kb;
@@ -113,13 +119,13 @@ __device__ __forceinline__ void bulk_copy_to_cluster(uint32_t dst_cluster, const
                  : "memory");
 }
 
-template <int ACT, bool HM>
-__global__ void __launch_bounds__(Umma2sCfgT<HM>::kThreads, 1)
+template <int ACT, bool HM, int BN_>
+__global__ void __launch_bounds__(Umma2sCfgT<HM, BN_>::kThreads, 1)
 gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                    __nv_bfloat16* __restrict__ Y,
                    const __nv_bfloat16* __restrict__ bias, int M, int N, int K, const __grid_constant__ Umma2sPlan plan,
                    int* __restrict__ status) {
-    using C = Umma2sCfgT<HM>;
+    using C = Umma2sCfgT<HM, BN_>;
     extern __shared__ uint8_t smem_raw[];
     Umma2sShared* sh = reinterpret_cast<Umma2sShared*>(smem_raw);
     const uint32_t ring_base = (ptx::smem_u32(smem_raw) + 256 + 1023) & ~1023u;
@@ -178,8 +184,8 @@ gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 ptx::mbar_arrive_expect_tx_cluster(full_leader, C::kStageBytes);
                 ptx::tma_load_2d_2cta(a_dst, &map_a, full_leader, kb * C::BK, tm * C::BM + hc * C::kRowsPerCta);
 #pragma unroll
-                for (int j = 0; j < 2; ++j)
-                    ptx::tma_load_2d_2cta(b_dst + j * C::kBChunkBytes, &map_b, full_leader, tn * C::BN + hc * 128 + j * 64,
+                for (int j = 0; j < C::kBChunks; ++j)
+                    ptx::tma_load_2d_2cta(b_dst + j * C::kBChunkBytes, &map_b, full_leader, tn * C::BN + hc * (C::BN / 2) + j * 64,
                                           kb * C::BK);
                 if (++s == C::kStages) { s = 0; ph ^= 1; }
             }
@@ -231,29 +237,30 @@ gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             ptx::umma_commit_2cta_local(&sh->drain);
             ptx::mbar_wait(&sh->drain, 0);
         }
-    } else if (S > 2) {
-        // ------------------------------------------------------------ epilogue warps, more than two bands
+    } else if (S > 2 || C::BN != 256) {
+        // ------------------------------------------------------------ epilogue warps, any number of bands and either tile width
         // Tensor-memory lane L of this CTA holds one row of the tile in its kTmemCols columns (256-row
-        // tiles: row L, columns 0..255; 128-row tiles: row L % 64, columns [128 (L / 64), +128)).  Band b
-        // finishes columns [keep b, keep b + keep) of every lane, keep = kTmemCols / S, and sends chunk d
-        // to the CTA of band d with the same h.  A share is 128 lanes x keep columns of fp32, float4
-        // index (column / 4) * 128 + lane; the ring holds S - 1 received shares, then S - 1 outgoing
-        // ones.  Of the two warps on a lane quarter each takes half of every chunk, 16 columns at a time.
+        // tiles: row L, all BN columns; 128-row tiles: row L % 64, columns [BN / 2 (L / 64), + BN / 2)).
+        // Band b finishes columns [keep b, keep b + keep) of every lane, keep = kTmemCols / S, and sends
+        // chunk d to the CTA of band d with the same h.  A share is 128 lanes x keep columns of fp32,
+        // float4 index (column / 4) * 128 + lane; the ring holds S - 1 received shares, then S - 1
+        // outgoing ones.  Of the two warps on a lane quarter each takes half of every chunk, 16 columns
+        // at a time (keep / 2 is a multiple of 16: the host plans no other split).
         constexpr int CT = C::kTmemCols;
         const int ew = warp - 2, q = warp & 3, ch = ew >> 2;
         const int L = q * 32 + lane;
-        const int keep = CT / S, W = keep / 2, ng = W / 16;        // 256-row tiles, S = 4: 64, 32, 2; 128-row tiles: 32, 16, 1
+        const int keep = CT / S, W = keep / 2, ng = W / 16;        // ng = 1 .. 4
         const uint32_t share_bytes = (uint32_t)(128 * keep * 4);
         const uint32_t recv_off = 0, send_off = (uint32_t)(S - 1) * share_bytes;
         const bool rows_live = (int64_t)tm * C::BM + hc * C::kRowsPerCta < M;
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
         const int64_t m = (int64_t)tm * C::BM + hc * C::kRowsPerCta + (HM ? (L & 63) : L);
-        const int64_t n0 = (int64_t)tn * C::BN + (HM ? (q >> 1) * 128 : 0) + band * keep + ch * W;   // first column of Y of this thread
+        const int64_t n0 = (int64_t)tn * C::BN + (HM ? (q >> 1) * (C::BN / 2) : 0) + band * keep + ch * W;   // first column of Y of this thread
         auto slot_of = [](int other, int self) { return other < self ? other : other - 1; };   // index among the S - 1 others
 
-        uint4 bias_w[2][2];                                 // fetched while the main loop runs
+        uint4 bias_w[4][2];                                 // fetched while the main loop runs
 #pragma unroll
-        for (int g = 0; g < 2; ++g)
+        for (int g = 0; g < 4; ++g)
 #pragma unroll
             for (int v = 0; v < 2; ++v) {
                 const int64_t n = n0 + g * 16 + v * 8;
@@ -266,58 +273,60 @@ gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         int site = 5;
         ptx::tcgen05_fence_after_sync();
 
-        if (ok && threadIdx.x == 64) {
-            for (int d = 0; d < S; ++d)
-                if (d != band) ptx::mbar_arrive_cluster(ptx::mapa_shared(ptx::smem_u32(&sh->partner_idle), (uint32_t)(2 * d + hc)));
-        }
-        if (ok && rows_live) {
-            for (int d = 0; d < S; ++d) {
-                if (d == band) continue;
-                float4* send = reinterpret_cast<float4*>(ring + send_off + (uint32_t)slot_of(d, band) * share_bytes) + L;
-                for (int g = 0; g < ng; ++g) {
-                    uint32_t r[16];
-                    ptx::tmem_ld_32x16(t_lane + d * keep + ch * W + g * 16, r);
-                    ptx::tmem_ld_wait();
-#pragma unroll
-                    for (int v = 0; v < 4; ++v)
-                        send[((ch * W + g * 16) / 4 + v) * 128] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
-                                                                              __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
-                }
+        if (S > 1) {
+            if (ok && threadIdx.x == 64) {
+                for (int d = 0; d < S; ++d)
+                    if (d != band) ptx::mbar_arrive_cluster(ptx::mapa_shared(ptx::smem_u32(&sh->partner_idle), (uint32_t)(2 * d + hc)));
             }
-            ptx::fence_proxy_async_smem();
-        }
-        umma2s_epi_bar_sync();
-        if (threadIdx.x == 64 && ok && rows_live) {
-            if (ptx::mbar_wait(&sh->partner_idle, 0)) {
+            if (ok && rows_live) {
                 for (int d = 0; d < S; ++d) {
                     if (d == band) continue;
-                    const uint32_t peer = (uint32_t)(2 * d + hc);
-                    bulk_copy_to_cluster(ptx::mapa_shared(ring_base + recv_off + (uint32_t)slot_of(band, d) * share_bytes, peer),
-                                         ring + send_off + (uint32_t)slot_of(d, band) * share_bytes, share_bytes,
-                                         ptx::mapa_shared(ptx::smem_u32(&sh->recv_full), peer));
+                    float4* send = reinterpret_cast<float4*>(ring + send_off + (uint32_t)slot_of(d, band) * share_bytes) + L;
+                    for (int g = 0; g < ng; ++g) {
+                        uint32_t r[16];
+                        ptx::tmem_ld_32x16(t_lane + d * keep + ch * W + g * 16, r);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int v = 0; v < 4; ++v)
+                            send[((ch * W + g * 16) / 4 + v) * 128] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                                                  __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                    }
                 }
-            } else {
-                site = 8;
+                ptx::fence_proxy_async_smem();
+            }
+            umma2s_epi_bar_sync();
+            if (threadIdx.x == 64 && ok && rows_live) {
+                if (ptx::mbar_wait(&sh->partner_idle, 0)) {
+                    for (int d = 0; d < S; ++d) {
+                        if (d == band) continue;
+                        const uint32_t peer = (uint32_t)(2 * d + hc);
+                        bulk_copy_to_cluster(ptx::mapa_shared(ring_base + recv_off + (uint32_t)slot_of(band, d) * share_bytes, peer),
+                                             ring + send_off + (uint32_t)slot_of(d, band) * share_bytes, share_bytes,
+                                             ptx::mapa_shared(ptx::smem_u32(&sh->recv_full), peer));
+                    }
+                } else {
+                    site = 8;
+                }
             }
         }
 
-        uint32_t racc[2][16];
-        if (ok && rows_live) {
-#pragma unroll
-            for (int g = 0; g < 2; ++g)
-                if (g < ng) ptx::tmem_ld_32x16(t_lane + band * keep + ch * W + g * 16, racc[g]);
+        // this warp's own first columns leave tensor memory while the partners' shares are on their way
+        uint32_t racc[16];
+        if (ok && rows_live) ptx::tmem_ld_32x16(t_lane + band * keep + ch * W, racc);
+        if (S > 1) {
+            if (ok && rows_live && !ptx::mbar_wait(&sh->recv_full, 0)) {
+                ok = false;
+                site = 9;
+            }
+            ok = __all_sync(0xffffffffu, ok);
         }
-        if (ok && rows_live && !ptx::mbar_wait(&sh->recv_full, 0)) {
-            ok = false;
-            site = 9;
-        }
-        ok = __all_sync(0xffffffffu, ok);
 
         if (ok && rows_live) {
-            ptx::tmem_ld_wait();
 #pragma unroll
-            for (int g = 0; g < 2; ++g) {
-                if (g >= ng) break;
+            for (int g = 0; g < 4; ++g) {
+                if (g >= ng) continue;                  // (no break: the loop stays unrolled and bias_w in registers)
+                if (g > 0) ptx::tmem_ld_32x16(t_lane + band * keep + ch * W + g * 16, racc);
+                ptx::tmem_ld_wait();
                 float x[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) x[i] = 0.0f;
@@ -325,7 +334,7 @@ gemm_umma2s_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                 for (int sb = 0; sb < S; ++sb) {
                     if (sb == band) {
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) x[i] += __uint_as_float(racc[g][i]);
+                        for (int i = 0; i < 16; ++i) x[i] += __uint_as_float(racc[i]);
                     } else {
                         const float4* recv = reinterpret_cast<const float4*>(ring + recv_off + (uint32_t)slot_of(sb, band) * share_bytes) + L;
                         float4 t[4];

@@ -7,6 +7,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -48,6 +49,7 @@ constexpr int64_t kOptionDefaults[OPTIML_OPT_COUNT] = {
     /* SKINNY_LATE_TRIGGER   */ 1,
     /* PAIR_SPLIT_MAX        */ 8,
     /* PAIR_HALF_HEIGHT      */ 1,
+    /* PAIR_TILE_WIDTH       */ 0,
 };
 
 // Streaming rates the skinny kernel's schedule is costed with (see launch_skinny_cfg).
@@ -190,16 +192,44 @@ bool variant_supports(optiml_handle_t h, int v, int64_t M, int64_t N, int64_t K,
 }
 
 // K slices (CTA pairs per tile) of the streaming pair kernel: as many as the device can hold
-// clusters for, with at least four K blocks per slice.
-int stream_split(optiml_handle_t h, int64_t tiles, int64_t num_kb) {
+// clusters for, with at least four K blocks per slice; a CTA must keep a multiple of 32
+// accumulator columns (its two epilogue warps per lane quarter work in pieces of 16).
+int stream_split(optiml_handle_t h, int64_t tiles, int64_t num_kb, int tmem_cols) {
     int split = 1;
     for (int i = 1; (1 << i) <= Umma2sCfg::kMaxSplit; ++i) {
         const int s = 1 << i;
-        if (tiles <= h->stream_clusters[i] && num_kb >= 4 * s) split = s;
+        if (tiles <= h->stream_clusters[i] && num_kb >= 4 * s && (tmem_cols / s) % 32 == 0) split = s;
     }
     const int64_t cap = h->options[OPTIML_OPT_PAIR_SPLIT_MAX];
     while (split > 1 && split > cap) split >>= 1;
     return split;
+}
+
+// Tile width of the streaming pair kernel.  What decides its time is how many bytes each SM has
+// to pull (its port takes about 90 GB/s) against the stream over B from HBM; 128-column tiles
+// double the number of CTAs where 256-column tiles are too few for the clusters the device
+// holds (N = 4096: 16 tiles, two pairs each = 64 CTAs; 32 narrow tiles = 128 CTAs) at the price
+// of reading A once more per column of tiles.
+int stream_tile_width(optiml_handle_t h, int64_t M, int64_t N, int64_t K, bool half_height) {
+    const int64_t cap = h->options[OPTIML_OPT_PAIR_TILE_WIDTH];
+    if (cap == 128 || cap == 256) return (int)cap;
+    const int bm = half_height ? 128 : 256, rows = bm / 2;
+    const int64_t tiles_m = ceil_div64(M, bm), num_kb = ceil_div64(K, 64);
+    double best = 0.0;
+    int width = 256;
+    for (int bn = 256; bn >= 128; bn -= 128) {
+        const int64_t tiles = tiles_m * ceil_div64(N, bn);
+        if (tiles > h->stream_clusters[0]) continue;
+        const int s = stream_split(h, tiles, num_kb, half_height ? bn / 2 : bn);
+        const double per_cta = (double)(rows + bn / 2) * 128.0 * (double)ceil_div64(num_kb, s);       // bytes through one SM's port
+        const double all = 2.0 * ((double)K * N + (double)M * K);
+        const double us = std::max(per_cta / 90e3, all / 6.3e6) + 5.0 + 1.0 * (s - 1);
+        if (best == 0.0 || us < best * 0.97) {       // the narrow form has to win by a margin
+            best = us;
+            width = bn;
+        }
+    }
+    return width;
 }
 
 // Whether the skinny kernel's schedule for this shape finishes every column tile in one CTA
@@ -485,14 +515,14 @@ optiml_status_t launch_umma2(optiml_handle_t h, const void* A, const void* B, co
 }
 
 // The streaming pair kernel: programmatic dependent launch plus a cluster of 2 * split CTAs.
-template <int ACT, bool HM>
+template <int ACT, bool HM, int BN>
 cudaError_t launch_umma2s_act(dim3 grid, int cluster, cudaStream_t st, const CUtensorMap& ma, const CUtensorMap& mb,
                               __nv_bfloat16* Y, const __nv_bfloat16* bias, int M, int N, int K,
                               const Umma2sPlan& plan, int* status) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
-    cfg.blockDim = dim3(Umma2sCfg::kThreads);
-    cfg.dynamicSmemBytes = Umma2sCfg::kSmemBytes;
+    cfg.blockDim = dim3(Umma2sCfgT<HM, BN>::kThreads);
+    cfg.dynamicSmemBytes = Umma2sCfgT<HM, BN>::kSmemBytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -503,16 +533,16 @@ cudaError_t launch_umma2s_act(dim3 grid, int cluster, cudaStream_t st, const CUt
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, gemm_umma2s_kernel<ACT, HM>, ma, mb, Y, bias, M, N, K, plan, status);
+    return cudaLaunchKernelEx(&cfg, gemm_umma2s_kernel<ACT, HM, BN>, ma, mb, Y, bias, M, N, K, plan, status);
 }
 
 // Up to 128 rows a pair shares a 128-row tile (64 rows per CTA); above, a 256-row tile.
 bool stream_half_height(optiml_handle_t h, int64_t M) { return M <= Umma2sHalfCfg::BM && h->options[OPTIML_OPT_PAIR_HALF_HEIGHT] != 0; }
 
-template <bool HM>
+template <bool HM, int BN>
 optiml_status_t launch_umma2s_form(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
                                    int K, int act, cudaStream_t st) {
-    using C = Umma2sCfgT<HM>;
+    using C = Umma2sCfgT<HM, BN>;
     CUtensorMap ma, mb;
     if (!get_map(h, &ma, A, (uint64_t)M, (uint64_t)K, C::kRowsPerCta, 64) || !get_map(h, &mb, B, (uint64_t)K, (uint64_t)N, 64, 64))
         return OPTIML_ERR_CUDA;
@@ -521,16 +551,17 @@ optiml_status_t launch_umma2s_form(optiml_handle_t h, const void* A, const void*
     plan.tiles_n = (int)ceil_div64(N, C::BN);
     plan.num_kb = (int)ceil_div64(K, C::BK);
     const int64_t tiles = (int64_t)plan.tiles_m * plan.tiles_n;
-    plan.split = stream_split(h, tiles, plan.num_kb);
-    if (h->log) fprintf(stderr, "[optiml] streaming pair plan: %d-row tiles=%lld split=%d kb=%d\n", C::BM, (long long)tiles, plan.split, plan.num_kb);
+    if (tiles > h->stream_clusters[0]) return OPTIML_ERR_UNSUPPORTED;
+    plan.split = stream_split(h, tiles, plan.num_kb, C::kTmemCols);
+    if (h->log) fprintf(stderr, "[optiml] streaming pair plan: %d x %d tiles=%lld split=%d kb=%d\n", C::BM, C::BN, (long long)tiles, plan.split, plan.num_kb);
     const int cluster = 2 * plan.split;
     const dim3 grid((unsigned)(tiles * cluster));
     const __nv_bfloat16* bi = (const __nv_bfloat16*)bias;
     switch (act) {
-    case OPTIML_ACT_RELU: launch_umma2s_act<kActRelu, HM>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
-    case OPTIML_ACT_GELU_TANH: launch_umma2s_act<kActGeluTanh, HM>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
-    case OPTIML_ACT_SIGMOID: launch_umma2s_act<kActSigmoid, HM>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
-    default: launch_umma2s_act<kActNone, HM>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
+    case OPTIML_ACT_RELU: launch_umma2s_act<kActRelu, HM, BN>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
+    case OPTIML_ACT_GELU_TANH: launch_umma2s_act<kActGeluTanh, HM, BN>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
+    case OPTIML_ACT_SIGMOID: launch_umma2s_act<kActSigmoid, HM, BN>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
+    default: launch_umma2s_act<kActNone, HM, BN>(grid, cluster, st, ma, mb, (__nv_bfloat16*)Y, bi, M, N, K, plan, h->status); break;
     }
     h->launches += 1;
     return cudaGetLastError() == cudaSuccess ? OPTIML_OK : OPTIML_ERR_CUDA;
@@ -538,8 +569,12 @@ optiml_status_t launch_umma2s_form(optiml_handle_t h, const void* A, const void*
 
 optiml_status_t launch_umma2s(optiml_handle_t h, const void* A, const void* B, const void* bias, void* Y, int M, int N,
                               int K, int act, cudaStream_t st) {
-    return stream_half_height(h, M) ? launch_umma2s_form<true>(h, A, B, bias, Y, M, N, K, act, st)
-                                    : launch_umma2s_form<false>(h, A, B, bias, Y, M, N, K, act, st);
+    const bool hm = stream_half_height(h, M);
+    const bool narrow = stream_tile_width(h, M, N, K, hm) == 128;
+    if (hm) return narrow ? launch_umma2s_form<true, 128>(h, A, B, bias, Y, M, N, K, act, st)
+                          : launch_umma2s_form<true, 256>(h, A, B, bias, Y, M, N, K, act, st);
+    return narrow ? launch_umma2s_form<false, 128>(h, A, B, bias, Y, M, N, K, act, st)
+                  : launch_umma2s_form<false, 256>(h, A, B, bias, Y, M, N, K, act, st);
 }
 
 // Clusters of `cluster` CTAs of the streaming pair kernel that can be resident at the same time.
@@ -556,7 +591,7 @@ int query_stream_clusters(int cluster) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_umma2s_kernel<kActNone, false>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_umma2s_kernel<kActNone, false, 256>, &cfg) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -587,14 +622,22 @@ bool configure_kernels() {
     ok &= set_smem(gemm_umma2_kernel<kActRelu>, Umma2Cfg::kSmemBytes);
     ok &= set_smem(gemm_umma2_kernel<kActGeluTanh>, Umma2Cfg::kSmemBytes);
     ok &= set_smem(gemm_umma2_kernel<kActSigmoid>, Umma2Cfg::kSmemBytes);
-    ok &= set_smem(gemm_umma2s_kernel<kActNone, false>, Umma2sCfg::kSmemBytes);
-    ok &= set_smem(gemm_umma2s_kernel<kActRelu, false>, Umma2sCfg::kSmemBytes);
-    ok &= set_smem(gemm_umma2s_kernel<kActGeluTanh, false>, Umma2sCfg::kSmemBytes);
-    ok &= set_smem(gemm_umma2s_kernel<kActSigmoid, false>, Umma2sCfg::kSmemBytes);
-    ok &= set_smem(gemm_umma2s_kernel<kActNone, true>, Umma2sHalfCfg::kSmemBytes);
-    ok &= set_smem(gemm_umma2s_kernel<kActRelu, true>, Umma2sHalfCfg::kSmemBytes);
-    ok &= set_smem(gemm_umma2s_kernel<kActGeluTanh, true>, Umma2sHalfCfg::kSmemBytes);
-    ok &= set_smem(gemm_umma2s_kernel<kActSigmoid, true>, Umma2sHalfCfg::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActNone, false, 256>, Umma2sCfgT<false, 256>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActRelu, false, 256>, Umma2sCfgT<false, 256>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActGeluTanh, false, 256>, Umma2sCfgT<false, 256>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActSigmoid, false, 256>, Umma2sCfgT<false, 256>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActNone, false, 128>, Umma2sCfgT<false, 128>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActRelu, false, 128>, Umma2sCfgT<false, 128>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActGeluTanh, false, 128>, Umma2sCfgT<false, 128>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActSigmoid, false, 128>, Umma2sCfgT<false, 128>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActNone, true, 256>, Umma2sCfgT<true, 256>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActRelu, true, 256>, Umma2sCfgT<true, 256>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActGeluTanh, true, 256>, Umma2sCfgT<true, 256>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActSigmoid, true, 256>, Umma2sCfgT<true, 256>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActNone, true, 128>, Umma2sCfgT<true, 128>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActRelu, true, 128>, Umma2sCfgT<true, 128>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActGeluTanh, true, 128>, Umma2sCfgT<true, 128>::kSmemBytes);
+    ok &= set_smem(gemm_umma2s_kernel<kActSigmoid, true, 128>, Umma2sCfgT<true, 128>::kSmemBytes);
     ok &= set_skinny(gemm_skinny_umma_kernel<16, 2>, SkinnyCfg<16, 2>::kSmemBytes);
     ok &= set_skinny(gemm_skinny_umma_kernel<16, 3>, SkinnyCfg<16, 3>::kSmemBytes);
     ok &= set_skinny(gemm_skinny_umma_kernel<32, 2>, SkinnyCfg<32, 2>::kSmemBytes);

@@ -134,6 +134,40 @@ def test_streaming_pair_variant_half_height_tiles(handle, M, N, K, act, split_ma
         handle.set_option(V.OPT_PAIR_HALF_HEIGHT, 1)
 
 
+@pytest.mark.parametrize("M,N,K", [(256, 128, 64),         # one narrow tile, one K block
+                                   (200, 520, 1096),       # 256-row tiles, ragged everywhere
+                                   (512, 392, 1032),       # two tile rows
+                                   (128, 264, 2048),       # 128-row tiles: 32 columns per lane half and CTA
+                                   (100, 776, 1096),
+                                   (64, 4096, 1024),       # 32 narrow tiles
+                                   (33, 136, 4096)])
+@pytest.mark.parametrize("act", [RELU, GELU])
+@pytest.mark.parametrize("split_max", [1, 2, 4])
+def test_streaming_pair_variant_narrow_tiles(handle, M, N, K, act, split_max):
+    """128-column tiles (64 columns of B per CTA), forced through the tile-width option, with one, two
+    and four CTA pairs per tile where the shape allows them."""
+    handle.set_option(V.OPT_PAIR_SPLIT_MAX, split_max)
+    handle.set_option(V.OPT_PAIR_TILE_WIDTH, 128)
+    try:
+        parity(handle, synth.make_case("c4", M=M, N=N, K=K, act=act), V.VARIANT_UMMA_2CTA_STREAM, "128-column tiles")
+    finally:
+        handle.set_option(V.OPT_PAIR_SPLIT_MAX, 8)
+        handle.set_option(V.OPT_PAIR_TILE_WIDTH, 0)
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 776, 1024), (384, 520, 2048), (100, 2056, 4096)])
+@pytest.mark.parametrize("width", [128, 256])
+def test_streaming_pair_variant_integer_inputs_either_width(handle, M, N, K, width):
+    handle.set_option(V.OPT_PAIR_TILE_WIDTH, width)
+    try:
+        c = synth.integer_case(M, N, K, BF16, RELU, seed=13)
+        handle.force_variant(V.VARIANT_UMMA_2CTA_STREAM)
+        bits, _ = H.run_case(handle, c)
+        H.check_bit_exact(bits, H.oracle_full(c), BF16, f"cluster kernel, {width}-column tiles, {M}x{N}x{K}")
+    finally:
+        handle.set_option(V.OPT_PAIR_TILE_WIDTH, 0)
+
+
 def test_streaming_pair_variant_refuses_more_tiles_than_clusters(handle):
     handle.force_variant(V.VARIANT_UMMA_2CTA_STREAM)
     c = synth.make_case("c4", M=2048, N=4096, K=64)          # 128 tiles
